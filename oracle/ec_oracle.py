@@ -1,0 +1,185 @@
+"""Plain fp64 CPU oracle of the expert-choice (EC) MoE feed-forward layer.
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT.  Slow and obvious on purpose: every
+function is the paper's definition written out with numpy in float64 (inputs
+are widened exactly; nothing is rounded in between), with no blocking, fusion
+or reordering.  Library primitives used as steps: numpy matmul, numpy stable
+argsort, scipy erf.
+
+Notation (Section 3.2): n tokens, d model width, d' hidden width, e experts,
+capacity factor c, k = n*c/e tokens per expert.  A "slot" is one (expert i,
+position j) pair; its flat id is i*k + j.
+
+Readings taken where the paper is silent (all listed in the design notes):
+softmax runs over the experts of one token (Section 3.4 says the gate models a
+distribution over experts); TopK breaks ties toward the lower token index and
+lists each expert's tokens by descending score; GeLU is the exact erf form by
+default (tanh form optional); no biases; G is used raw (no renormalisation);
+a token chosen by no expert gets a zero output row; in the backward pass the
+index matrix I is a constant, so the gate is trained through G only.
+
+Every function here is pinned by tests/test_oracle_*.py against closed forms,
+brute force, invariants, library routines and finite differences; nothing in
+this file is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+from scipy.special import erf as _erf
+
+F64 = np.float64
+
+
+def capacity(n: int, c: float, e: int) -> int:
+    """Eq. 1: k = n*c/e.  Non-integer values are floored; k < 1 or k > n is an error."""
+    k = int(math.floor(n * float(c) / e + 1e-9))
+    if k < 1 or k > n:
+        raise ValueError(f"capacity k={k} outside [1, n={n}]")
+    return k
+
+
+def gate(X, Wg):
+    """Eq. 2, first line: S = Softmax(X . Wg), one distribution over the e experts per token."""
+    L = np.asarray(X, F64) @ np.asarray(Wg, F64)
+    L = L - L.max(axis=1, keepdims=True)
+    P = np.exp(L)
+    return P / P.sum(axis=1, keepdims=True)
+
+
+def topk(S, k: int):
+    """Eq. 2, second line: G, I = TopK(S^T, k).
+
+    For expert i the tokens are ordered by score S[t, i] descending, equal
+    scores by ascending t (a stable sort of the negated column); the first k
+    are I[i, :], and G[i, j] = S[I[i, j], i].
+    """
+    S = np.asarray(S)
+    n, e = S.shape
+    I = np.empty((e, k), np.int64)
+    G = np.empty((e, k), S.dtype)
+    for i in range(e):
+        order = np.argsort(-S[:, i], kind="stable")
+        I[i] = order[:k]
+        G[i] = S[I[i], i]
+    return G, I
+
+
+def inverse_index(I, n: int):
+    """Index form of P = Onehot(I) (Eq. 2) read by token: for token t, the flat
+    slot ids i*k+j with I[i, j] = t, in ascending order (hence ascending expert).
+    Returns row_ptr [n+1] and slots [e*k]."""
+    I = np.asarray(I)
+    e, k = I.shape
+    flat = I.reshape(-1)
+    order = np.argsort(flat, kind="stable")          # ascending token, then ascending slot id
+    counts = np.bincount(flat, minlength=n)
+    row_ptr = np.zeros(n + 1, np.int64)
+    row_ptr[1:] = np.cumsum(counts)
+    return row_ptr, order.astype(np.int64)
+
+
+def gelu(z, variant: str = "erf"):
+    """GeLU(z) = z * Phi(z) (erf form), or its tanh approximation."""
+    z = np.asarray(z, F64)
+    if variant == "erf":
+        return 0.5 * z * (1.0 + _erf(z / math.sqrt(2.0)))
+    if variant == "tanh":
+        return 0.5 * z * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (z + 0.044715 * z ** 3)))
+    raise ValueError(variant)
+
+
+def gelu_grad(z, variant: str = "erf"):
+    """d GeLU / dz."""
+    z = np.asarray(z, F64)
+    if variant == "erf":
+        Phi = 0.5 * (1.0 + _erf(z / math.sqrt(2.0)))
+        phi = np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+        return Phi + z * phi
+    if variant == "tanh":
+        a = math.sqrt(2.0 / math.pi)
+        u = a * (z + 0.044715 * z ** 3)
+        th = np.tanh(u)
+        return 0.5 * (1.0 + th) + 0.5 * z * (1.0 - th * th) * a * (1.0 + 3 * 0.044715 * z * z)
+    raise ValueError(variant)
+
+
+def route(X, Wg, c: float, S_override=None):
+    """Eq. 1-2: S, G, I and the token->slot inverse index."""
+    n = np.asarray(X).shape[0]
+    e = np.asarray(Wg).shape[1]
+    k = capacity(n, c, e)
+    S = gate(X, Wg) if S_override is None else np.asarray(S_override, F64)
+    G, I = topk(S, k)
+    row_ptr, slots = inverse_index(I, n)
+    return dict(k=k, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots)
+
+
+def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None):
+    """Eq. 1-4.  Returns every intermediate.
+
+    S_override replaces the gate output (the routing is then taken from it);
+    I_override additionally fixes the index matrix (G is read from S at I).
+    Both exist so that later stages can be compared on identical routing.
+    """
+    X = np.asarray(X, F64); Wg = np.asarray(Wg, F64)
+    W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
+    n, d = X.shape
+    e = Wg.shape[1]
+    r = route(X, Wg, c, S_override)
+    k, S = r["k"], r["S"]
+    if I_override is not None:
+        I = np.asarray(I_override, np.int64)
+        G = np.stack([S[I[i], i] for i in range(e)])
+        row_ptr, slots = inverse_index(I, n)
+        r.update(I=I, G=G, row_ptr=row_ptr, slots=slots)
+    I, G = r["I"], r["G"]
+    X_in = X[I]                                            # Eq. 3: X_in = P . X,  [e, k, d]
+    Z = np.stack([X_in[i] @ W1[i] for i in range(e)])      # [e, k, d']
+    H = gelu(Z, gelu_variant)
+    X_e = np.stack([H[i] @ W2[i].T for i in range(e)])     # [e, k, d]
+    X_out = np.zeros((n, d), F64)                          # Eq. 4, experts in ascending order
+    for i in range(e):
+        for j in range(k):
+            X_out[I[i, j]] += G[i, j] * X_e[i, j]
+    r.update(X_in=X_in, Z=Z, H=H, X_e=X_e, X_out=X_out)
+    return r
+
+
+def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf"):
+    """Gradients of <dX_out, X_out> with respect to X, Wg, W1, W2 by the chain rule
+    through Eq. 4, 3, 2 in that order, with I held constant."""
+    X = np.asarray(X, F64); Wg = np.asarray(Wg, F64)
+    W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
+    dX_out = np.asarray(dX_out, F64)
+    n, d = X.shape
+    e = Wg.shape[1]
+    S, G, I = fwd["S"], fwd["G"], fwd["I"]
+    X_in, Z, H, X_e = fwd["X_in"], fwd["Z"], fwd["H"], fwd["X_e"]
+    k = I.shape[1]
+    dY = dX_out[I]                                         # [e, k, d] rows of dX_out seen by each slot
+    dX_e = G[:, :, None] * dY                              # Eq. 4 w.r.t. X_e
+    dG = np.einsum("ijd,ijd->ij", dY, X_e)                 # Eq. 4 w.r.t. G
+    dH = np.stack([dX_e[i] @ W2[i] for i in range(e)])     # [e, k, d']
+    dW2 = np.stack([dX_e[i].T @ H[i] for i in range(e)])   # [e, d, d']
+    dZ = dH * gelu_grad(Z, gelu_variant)
+    dW1 = np.stack([X_in[i].T @ dZ[i] for i in range(e)])  # [e, d, d']
+    dX_in = np.stack([dZ[i] @ W1[i].T for i in range(e)])  # [e, k, d]
+    dS = np.zeros((n, e), F64)
+    for i in range(e):
+        dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
+    dL = S * (dS - (dS * S).sum(axis=1, keepdims=True))    # softmax Jacobian, per token row
+    dWg = X.T @ dL
+    dX = dL @ Wg.T
+    for i in range(e):
+        for j in range(k):
+            dX[I[i, j]] += dX_in[i, j]
+    return dict(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2, dX_e=dX_e, dG=dG, dH=dH, dZ=dZ,
+                dX_in=dX_in, dS=dS, dL=dL)
+
+
+def experts_per_token(row_ptr):
+    """Number of experts that chose each token (the quantity of Fig. 3)."""
+    row_ptr = np.asarray(row_ptr)
+    return row_ptr[1:] - row_ptr[:-1]
