@@ -1,0 +1,144 @@
+/*
+ * ecmoe.h - C ABI of the expert-choice (EC) mixture-of-experts feed-forward layer
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the one of "Mixture-of-Experts with Expert Choice Routing"
+ * (arXiv 2202.09368), Section 3.2.  Notation follows the paper: n tokens in the
+ * routed group, d model width, d' hidden width of an expert, e experts, capacity
+ * factor c, k = n*c/e tokens per expert (Eq. 1).  A "slot" is one (expert i,
+ * position j) pair; its flat id is i*k + j and there are e*k of them.
+ *
+ * Conventions for every entry point unless it says otherwise
+ *  - Tensor arguments are DEVICE pointers owned by the caller, dense row-major,
+ *    16-byte aligned.  The library never allocates, frees or keeps device memory.
+ *  - Work is queued on `cuda_stream` (a cudaStream_t passed as void*; NULL is the
+ *    legacy default stream) and the call returns without synchronising; results
+ *    are valid once the caller has synchronised that stream.
+ *  - `ws` is scratch of at least ec_workspace_bytes(cfg) bytes, 256-byte aligned;
+ *    its contents are undefined after a call.  Two calls that overlap on the GPU
+ *    must not share a workspace.
+ *  - Errors are return codes.  Arguments are checked on the host before anything
+ *    is launched; nothing is launched when the code is not EC_OK.
+ *  - X, Wg, W1, W2, X_out, dX_out and all gradients have the element type
+ *    cfg->dtype; S and G are always fp32 and index outputs are int32.
+ *  - Restrictions (EC_ERR_UNSUPPORTED otherwise): d_model and d_ff rows must be a
+ *    multiple of 16 bytes long; n < 2^31; 1 <= E <= 256; E*k < 2^31; groups == 1.
+ */
+#ifndef ECMOE_H_
+#define ECMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  EC_OK = 0,
+  EC_ERR_INVALID_ARG = 1, /* null pointer, misaligned pointer, k outside [1, n], bad enum        */
+  EC_ERR_UNSUPPORTED = 2, /* a documented restriction is violated                                */
+  EC_ERR_WORKSPACE = 3,   /* ws_bytes or saved_bytes smaller than required                       */
+  EC_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (launch, tensor-map encode)    */
+  EC_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported by ec_read_status)     */
+} ec_status;
+
+typedef enum { EC_F32 = 0, EC_BF16 = 1 } ec_dtype;
+typedef enum { EC_GELU_ERF = 0, EC_GELU_TANH = 1 } ec_gelu;
+
+/* One layer call.  Plain data, passed by pointer, never retained. */
+typedef struct {
+  int64_t n;       /* tokens in the group (Section 3.2: batch size x sequence length) */
+  int32_t d_model; /* d                                                               */
+  int32_t d_ff;    /* d'                                                              */
+  int32_t E;       /* number of experts e                                             */
+  int32_t groups;  /* independent routing groups; must be 1                           */
+  double c;        /* capacity factor (Eq. 1)                                         */
+  int32_t dtype;   /* ec_dtype                                                        */
+  int32_t gelu;    /* ec_gelu                                                         */
+} ec_config;
+
+/* Views into the forward->backward blob (device pointers), for inspection and tests. */
+typedef struct {
+  float* S;         /* [n, E]     gate scores (Eq. 2)                                  */
+  int32_t* I;       /* [E, k]     token chosen for each slot                           */
+  float* G;         /* [E, k]     gate weight of each slot, G[i,j] = S[I[i,j], i]      */
+  int32_t* row_ptr; /* [n+1]      token -> range in `slots`                            */
+  int32_t* slots;   /* [E*k]      flat slot ids of each token, ascending               */
+  void* X_in;       /* [E, k, d]  gathered expert inputs (Eq. 3)                       */
+  void* Z;          /* [E, k, d'] X_in[i] . W1[i]                                      */
+  void* H;          /* [E, k, d'] GeLU(Z)                                              */
+  void* X_e;        /* [E, k, d]  expert outputs H[i] . W2[i]^T                        */
+} ec_saved_ptrs;
+
+/* Eq. 1: k = floor(n*c/E).  Returns -1 when cfg is NULL or k falls outside [1, n]. */
+int64_t ec_capacity(const ec_config* cfg);
+
+/* Bytes of scratch every call below needs (the maximum over the three).  0 on a bad cfg. */
+size_t ec_workspace_bytes(const ec_config* cfg);
+
+/* Bytes of the blob ec_moe_forward fills for ec_moe_backward.  0 on a bad cfg. */
+size_t ec_saved_bytes(const ec_config* cfg);
+
+/* Computes the addresses of the blob's parts.  Host-only arithmetic; `saved` is not touched. */
+ec_status ec_saved_view(const ec_config* cfg, void* saved, ec_saved_ptrs* out);
+
+/*
+ * Routing, Eq. 1-2: S = Softmax(X . Wg) over the E experts of each token, then for
+ * every expert the k largest entries of its column of S.  Ties go to the lower
+ * token index; each expert's slots are listed by descending score (equal scores
+ * by ascending token), which makes I and G unique.  Also emits the index form of
+ * P = Onehot(I) read by token: slots[row_ptr[t] .. row_ptr[t+1]) are the flat
+ * slot ids that hold token t, ascending (so ascending expert).
+ *   X [n, d], Wg [d, E] in;  S [n, E], I [E, k], G [E, k], row_ptr [n+1], slots [E*k] out.
+ * On the bf16 path logits are accumulated in fp32 and the softmax and the
+ * comparison run on fp32 values.
+ */
+ec_status ec_route(const ec_config* cfg, const void* X, const void* Wg, float* S, int32_t* I,
+                   float* G, int32_t* row_ptr, int32_t* slots, void* ws, size_t ws_bytes,
+                   void* cuda_stream);
+
+/*
+ * Forward, Eq. 2-4: routing as above, X_in = P . X (gather), X_e[i] =
+ * GeLU(X_in[i] . W1[i]) . W2[i]^T for every expert, and X_out[t, :] = sum over the
+ * slots (i, j) holding t of G[i, j] * X_e[i, j, :], experts in ascending order, in
+ * fp32, rounded once.  Rows of tokens that no expert chose are zero.
+ *   W1, W2 [E, d, d'] (W2 is applied transposed);  X_out [n, d] out.
+ * `saved` (ec_saved_bytes(cfg) bytes, 256-byte aligned) receives what the backward
+ * pass needs; it must always be given (the intermediates live there).
+ */
+ec_status ec_moe_forward(const ec_config* cfg, const void* X, const void* Wg, const void* W1,
+                         const void* W2, void* X_out, void* saved, size_t saved_bytes, void* ws,
+                         size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Backward of Eq. 2-4 (the paper trains the gate, Section 3.4, and leaves the
+ * derivative to automatic differentiation): gradients of <dX_out, X_out> with I held
+ * constant, so the gate receives gradient through G only.
+ *   dX_out [n, d] in, `saved` as filled by ec_moe_forward with the same cfg and inputs;
+ *   dX [n, d], dWg [d, E], dW1, dW2 [E, d, d'] out, overwritten (not accumulated).
+ */
+ec_status ec_moe_backward(const ec_config* cfg, const void* X, const void* Wg, const void* W1,
+                          const void* W2, const void* dX_out, const void* saved,
+                          size_t saved_bytes, void* dX, void* dWg, void* dW1, void* dW2, void* ws,
+                          size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and reads the status word the kernels of the last call
+ * on `ws` left there: EC_OK, or EC_ERR_TIMEOUT when a bounded wait inside a kernel
+ * gave up (the outputs of that call are then undefined), or EC_ERR_CUDA when the
+ * stream reports an error.
+ */
+ec_status ec_read_status(const void* ws, void* cuda_stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char* ec_status_string(ec_status s);
+
+/* 1 if the bf16 path of this cfg runs its expert GEMMs on the tcgen05 tensor-core
+ * kernels, 0 if it falls back to the plain FMA kernels (fp32 path, odd shapes). */
+int ec_uses_tensor_cores(const ec_config* cfg);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECMOE_H_ */

@@ -1,0 +1,202 @@
+"""Thin ctypes binding of libecmoe.so (see include/ecmoe.h).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA
+kernels.  torch is used to own device memory and to name the current stream.
+There is no fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libecmoe.so")
+_lib = None
+
+EC_OK, EC_ERR_INVALID_ARG, EC_ERR_UNSUPPORTED, EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT = range(6)
+EC_F32, EC_BF16 = 0, 1
+EC_GELU_ERF, EC_GELU_TANH = 0, 1
+
+EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
+           "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
+           "ec_uses_tensor_cores"]
+
+
+class ec_config(C.Structure):
+    _fields_ = [("n", C.c_int64), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32),
+                ("groups", C.c_int32), ("c", C.c_double), ("dtype", C.c_int32), ("gelu", C.c_int32)]
+
+
+class ec_saved_ptrs(C.Structure):
+    _fields_ = [(name, C.c_void_p) for name in
+                ("S", "I", "G", "row_ptr", "slots", "X_in", "Z", "H", "X_e")]
+
+
+class EcError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} ({code})")
+
+
+def lib():
+    """Loads the library once.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2202_09368_b200.build`; "
+                               "there is no fallback path")
+        L = C.CDLL(_LIB_PATH)
+        P, V = C.POINTER(ec_config), C.c_void_p
+        L.ec_capacity.restype = C.c_int64; L.ec_capacity.argtypes = [P]
+        L.ec_workspace_bytes.restype = C.c_size_t; L.ec_workspace_bytes.argtypes = [P]
+        L.ec_saved_bytes.restype = C.c_size_t; L.ec_saved_bytes.argtypes = [P]
+        L.ec_saved_view.restype = C.c_int; L.ec_saved_view.argtypes = [P, V, C.POINTER(ec_saved_ptrs)]
+        L.ec_route.restype = C.c_int
+        L.ec_route.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V]
+        L.ec_moe_forward.restype = C.c_int
+        L.ec_moe_forward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, C.c_size_t, V]
+        L.ec_moe_backward.restype = C.c_int
+        L.ec_moe_backward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, V, V, V, V, C.c_size_t, V]
+        L.ec_read_status.restype = C.c_int; L.ec_read_status.argtypes = [V, V]
+        L.ec_status_string.restype = C.c_char_p; L.ec_status_string.argtypes = [C.c_int]
+        L.ec_uses_tensor_cores.restype = C.c_int; L.ec_uses_tensor_cores.argtypes = [P]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().ec_status_string(code).decode()
+
+
+def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=1) -> ec_config:
+    dt = {torch.float32: EC_F32, torch.bfloat16: EC_BF16}[dtype]
+    return ec_config(int(n), int(d_model), int(d_ff), int(E), int(groups), float(c), dt,
+                     {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu])
+
+
+def ec_capacity(cfg: ec_config) -> int:
+    return int(lib().ec_capacity(C.byref(cfg)))
+
+
+def ec_workspace_bytes(cfg: ec_config) -> int:
+    return int(lib().ec_workspace_bytes(C.byref(cfg)))
+
+
+def ec_saved_bytes(cfg: ec_config) -> int:
+    return int(lib().ec_saved_bytes(C.byref(cfg)))
+
+
+def ec_uses_tensor_cores(cfg: ec_config) -> bool:
+    return bool(lib().ec_uses_tensor_cores(C.byref(cfg)))
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _torch_dtype(cfg):
+    return torch.float32 if cfg.dtype == EC_F32 else torch.bfloat16
+
+
+def _check(code, what):
+    if code != EC_OK:
+        raise EcError(code, what)
+
+
+def alloc_workspace(cfg, device="cuda") -> torch.Tensor:
+    nb = ec_workspace_bytes(cfg)
+    if nb == 0:
+        raise EcError(EC_ERR_INVALID_ARG, "ec_workspace_bytes")
+    return torch.empty(nb, dtype=torch.uint8, device=device)
+
+
+def alloc_saved(cfg, device="cuda") -> torch.Tensor:
+    nb = ec_saved_bytes(cfg)
+    if nb == 0:
+        raise EcError(EC_ERR_INVALID_ARG, "ec_saved_bytes")
+    return torch.empty(nb, dtype=torch.uint8, device=device)
+
+
+@dataclass
+class Routing:
+    S: torch.Tensor
+    I: torch.Tensor
+    G: torch.Tensor
+    row_ptr: torch.Tensor
+    slots: torch.Tensor
+
+
+def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
+    """Eq. 1-2 on device tensors; returns S, I, G and the token->slot index."""
+    k = ec_capacity(cfg)
+    if k < 1:
+        raise EcError(EC_ERR_INVALID_ARG, "ec_capacity")
+    dev = X.device
+    if out is None:
+        out = Routing(torch.empty(cfg.n, cfg.E, dtype=torch.float32, device=dev),
+                      torch.empty(cfg.E, k, dtype=torch.int32, device=dev),
+                      torch.empty(cfg.E, k, dtype=torch.float32, device=dev),
+                      torch.empty(cfg.n + 1, dtype=torch.int32, device=dev),
+                      torch.empty(cfg.E * k, dtype=torch.int32, device=dev))
+    ws = alloc_workspace(cfg, dev) if ws is None else ws
+    _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
+                          _ptr(out.row_ptr), _ptr(out.slots), _ptr(ws), ws.numel(), _stream()), "ec_route")
+    return out
+
+
+def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None):
+    """Eq. 2-4.  Returns (X_out, saved)."""
+    dev = X.device
+    X_out = torch.empty(cfg.n, cfg.d_model, dtype=_torch_dtype(cfg), device=dev) if X_out is None else X_out
+    saved = alloc_saved(cfg, dev) if saved is None else saved
+    ws = alloc_workspace(cfg, dev) if ws is None else ws
+    _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),
+                                _ptr(saved), saved.numel(), _ptr(ws), ws.numel(), _stream()), "ec_moe_forward")
+    return X_out, saved
+
+
+def ec_moe_backward(cfg, X, Wg, W1, W2, dX_out, saved, grads=None, ws=None):
+    """Backward of Eq. 2-4.  Returns (dX, dWg, dW1, dW2)."""
+    dev = X.device
+    if grads is None:
+        grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
+    dX, dWg, dW1, dW2 = grads
+    ws = alloc_workspace(cfg, dev) if ws is None else ws
+    _check(lib().ec_moe_backward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(dX_out),
+                                 _ptr(saved), saved.numel(), _ptr(dX), _ptr(dWg), _ptr(dW1), _ptr(dW2),
+                                 _ptr(ws), ws.numel(), _stream()), "ec_moe_backward")
+    return dX, dWg, dW1, dW2
+
+
+def ec_read_status(ws) -> int:
+    return int(lib().ec_read_status(_ptr(ws), _stream()))
+
+
+def saved_view(cfg, saved) -> dict:
+    """Torch views of the parts of the forward->backward blob (no copies)."""
+    v = ec_saved_ptrs()
+    _check(lib().ec_saved_view(C.byref(cfg), _ptr(saved), C.byref(v)), "ec_saved_view")
+    k = ec_capacity(cfg)
+    base = saved.data_ptr()
+    dt = _torch_dtype(cfg)
+    es = 4 if cfg.dtype == EC_F32 else 2
+
+    def view(addr, shape, dtype, esz):
+        cnt = 1
+        for s in shape:
+            cnt *= s
+        off = addr - base
+        return saved[off:off + cnt * esz].view(dtype).view(*shape)
+
+    n, E, d, f = cfg.n, cfg.E, cfg.d_model, cfg.d_ff
+    return dict(S=view(v.S, (n, E), torch.float32, 4), I=view(v.I, (E, k), torch.int32, 4),
+                G=view(v.G, (E, k), torch.float32, 4), row_ptr=view(v.row_ptr, (n + 1,), torch.int32, 4),
+                slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es),
+                Z=view(v.Z, (E, k, f), dt, es), H=view(v.H, (E, k, f), dt, es),
+                X_e=view(v.X_e, (E, k, d), dt, es))

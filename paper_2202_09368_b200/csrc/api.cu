@@ -1,0 +1,288 @@
+// C ABI of the expert-choice MoE layer: argument checks, workspace carving and the sequence of
+// kernel launches for routing (Eq. 1-2), forward (Eq. 2-4) and backward.
+#include "../../include/ecmoe.h"
+#include "internal.h"
+
+#include <math.h>
+#include <string.h>
+
+using namespace ecmoe;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t up(size_t b) { return (b + kAlign - 1) & ~(kAlign - 1); }
+inline size_t esize(int dtype) { return dtype == EC_F32 ? 4 : 2; }
+
+struct Dims { int64_t n, k, slots; int d, dff, E; int dtype, gelu; size_t eb; };
+
+ec_status check_cfg(const ec_config* c, Dims* D) {
+  if (!c) return EC_ERR_INVALID_ARG;
+  if (c->dtype != EC_F32 && c->dtype != EC_BF16) return EC_ERR_INVALID_ARG;
+  if (c->gelu != EC_GELU_ERF && c->gelu != EC_GELU_TANH) return EC_ERR_INVALID_ARG;
+  if (c->n < 1 || c->d_model < 1 || c->d_ff < 1 || c->E < 1 || !(c->c > 0.0)) return EC_ERR_INVALID_ARG;
+  if (c->groups != 1) return EC_ERR_UNSUPPORTED;
+  if (c->n >= ((int64_t)1 << 31) || c->E > 256) return EC_ERR_UNSUPPORTED;
+  const size_t eb = esize(c->dtype);
+  if ((c->d_model * eb) % 16 || (c->d_ff * eb) % 16) return EC_ERR_UNSUPPORTED;
+  const int64_t k = ec_capacity(c);
+  if (k < 1) return EC_ERR_INVALID_ARG;
+  if ((int64_t)c->E * k >= ((int64_t)1 << 31)) return EC_ERR_UNSUPPORTED;
+  if (D) { D->n = c->n; D->k = k; D->slots = (int64_t)c->E * k; D->d = c->d_model; D->dff = c->d_ff;
+           D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb; }
+  return EC_OK;
+}
+
+struct SavedLayout { size_t S, I, G, row_ptr, slots, X_in, Z, H, X_e, total; };
+SavedLayout saved_layout(const Dims& D) {
+  SavedLayout L; size_t o = 0;
+  auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
+  L.S = take((size_t)D.n * D.E * 4);
+  L.I = take((size_t)D.slots * 4);
+  L.G = take((size_t)D.slots * 4);
+  L.row_ptr = take((size_t)(D.n + 1) * 4);
+  L.slots = take((size_t)D.slots * 4);
+  L.X_in = take((size_t)D.slots * D.d * D.eb);
+  L.Z = take((size_t)D.slots * D.dff * D.eb);
+  L.H = take((size_t)D.slots * D.dff * D.eb);
+  L.X_e = take((size_t)D.slots * D.d * D.eb);
+  L.total = o;
+  return L;
+}
+
+int dwg_splits(const Dims& D) { int64_t p = (D.n + 1023) / 1024; return (int)(p < 1 ? 1 : (p > 32 ? 32 : p)); }
+
+struct WsLayout { size_t status, topk, inverse, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
+WsLayout ws_layout(const Dims& D) {
+  WsLayout L; size_t o = 0;
+  auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
+  L.status = take(sizeof(StatusWord));
+  const size_t base = o;
+  L.topk = take(topk_scratch_bytes(D.n, D.E, D.k));
+  L.inverse = take(inverse_scratch_bytes(D.n));
+  const size_t fwd_end = o;
+  o = base;                                   // the backward pass reuses the same region
+  L.dX_e = take((size_t)D.slots * D.d * D.eb);
+  L.dG = take((size_t)D.slots * 4);
+  L.dZ = take((size_t)D.slots * D.dff * D.eb);
+  L.dX_in = take((size_t)D.slots * D.d * D.eb);
+  L.dL = take((size_t)D.n * D.E * 4);
+  L.dWg_part = take((size_t)dwg_splits(D) * D.d * D.E * 4);
+  L.total = o > fwd_end ? o : fwd_end;
+  return L;
+}
+
+inline bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
+
+#define EC_CUDA(x) do { if ((x) != cudaSuccess) return EC_ERR_CUDA; } while (0)
+
+// One expert-batched GEMM: tensor cores when the shape allows, FMA otherwise.
+struct BatchedGemm {
+  const void* A; int a_mn; int64_t lda, batch_a;     // a_mn = 0: A stored [M][K]; 1: stored [K][M]
+  const void* B; int b_mn; int64_t ldb, batch_b;     // b_mn = 0: B stored [N][K]; 1: stored [K][N]
+  void* C; int64_t ldc, batch_c;
+  int M, N, K, batches, epi;
+  void* C2; const void* Zin;
+};
+
+ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaStream_t st) {
+  if (D.dtype == EC_BF16) {
+    TcGemmArgs t; memset(&t, 0, sizeof(t));
+    t.A = b.A; t.B = b.B; t.a_mn_major = b.a_mn; t.b_mn_major = b.b_mn;
+    t.M = b.M; t.N = b.N; t.K = b.K; t.batches = b.batches;
+    t.lda = b.lda; t.ldb = b.ldb; t.batch_a = b.batch_a; t.batch_b = b.batch_b;
+    t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c;
+    t.status = status_word;
+    if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); return EC_OK; }
+  }
+  GemmArgs g; memset(&g, 0, sizeof(g));
+  g.A = b.A; g.B = b.B; g.C = b.C; g.a_dtype = g.b_dtype = g.c_dtype = D.dtype;
+  g.M = b.M; g.N = b.N; g.K = b.K; g.batches = b.batches;
+  g.sam = b.a_mn ? 1 : b.lda; g.sak = b.a_mn ? b.lda : 1;
+  g.sbk = b.b_mn ? b.ldb : 1; g.sbn = b.b_mn ? 1 : b.ldb;
+  g.ldc = b.ldc; g.batch_a = b.batch_a; g.batch_b = b.batch_b; g.batch_c = b.batch_c;
+  g.epi = b.epi; g.gelu = D.gelu; g.C2 = b.C2; g.Zin = b.Zin;
+  EC_CUDA(launch_gemm_simt(g, st));
+  return EC_OK;
+}
+
+ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int32_t* I, float* G,
+                     int32_t* row_ptr, int32_t* slots, char* ws, const WsLayout& W, cudaStream_t st) {
+  bool done = false;
+  if (D.dtype == EC_BF16) {
+    TcGemmArgs t; memset(&t, 0, sizeof(t));
+    t.A = X; t.B = Wg; t.a_mn_major = 0; t.b_mn_major = 1;
+    t.M = (int)D.n; t.N = D.E; t.K = D.d; t.batches = 1; t.lda = D.d; t.ldb = D.E;
+    t.epi = EPI_SOFTMAX; t.S = S; t.ldc = D.E; t.status = (int*)(ws + W.status);
+    if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); done = true; }
+  }
+  if (!done) EC_CUDA(launch_gate_softmax_simt(D.dtype, X, Wg, S, D.n, D.d, D.E, st));
+  EC_CUDA(launch_topk(S, D.n, D.E, D.k, I, G, ws + W.topk, st));
+  EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
+  return EC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t ec_capacity(const ec_config* c) {
+  if (!c || c->E < 1 || c->n < 1 || !(c->c > 0.0)) return -1;
+  const double kd = floor((double)c->n * c->c / (double)c->E + 1e-9);
+  if (kd < 1.0 || kd > (double)c->n) return -1;
+  return (int64_t)kd;
+}
+
+size_t ec_workspace_bytes(const ec_config* c) {
+  Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
+  return ws_layout(D).total;
+}
+
+size_t ec_saved_bytes(const ec_config* c) {
+  Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
+  return saved_layout(D).total;
+}
+
+ec_status ec_saved_view(const ec_config* c, void* saved, ec_saved_ptrs* out) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!saved || !out) return EC_ERR_INVALID_ARG;
+  const SavedLayout L = saved_layout(D); char* b = (char*)saved;
+  out->S = (float*)(b + L.S); out->I = (int32_t*)(b + L.I); out->G = (float*)(b + L.G);
+  out->row_ptr = (int32_t*)(b + L.row_ptr); out->slots = (int32_t*)(b + L.slots);
+  out->X_in = b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = b + L.X_e;
+  return EC_OK;
+}
+
+ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, int32_t* I, float* G,
+                   int32_t* row_ptr, int32_t* slots, void* ws, size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X || !Wg || !S || !I || !G || !row_ptr || !slots || !ws) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(S, 16) || misaligned(I, 16) || misaligned(G, 16) ||
+      misaligned(row_ptr, 16) || misaligned(slots, 16) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D);
+  if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
+}
+
+ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, const void* W1, const void* W2,
+                         void* X_out, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X || !Wg || !W1 || !W2 || !X_out || !saved || !ws) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(W1, 16) || misaligned(W2, 16) || misaligned(X_out, 16) ||
+      misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D);
+  if (ws_bytes < W.total || saved_bytes < L.total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* sv = (char*)saved; char* w = (char*)ws;
+  float* S = (float*)(sv + L.S); int32_t* I = (int32_t*)(sv + L.I); float* G = (float*)(sv + L.G);
+  int32_t* row_ptr = (int32_t*)(sv + L.row_ptr); int32_t* slots = (int32_t*)(sv + L.slots);
+  void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; void* X_e = sv + L.X_e;
+  int* status = (int*)(w + W.status);
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st)) != EC_OK) return s;
+  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
+  const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
+  // Z = X_in[i] . W1[i],  H = GeLU(Z)
+  BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr};
+  if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
+  // X_e = H[i] . W2[i]^T
+  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
+  if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
+  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
+  return EC_OK;
+}
+
+ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, const void* W1, const void* W2,
+                          const void* dX_out, const void* saved, size_t saved_bytes, void* dX, void* dWg,
+                          void* dW1, void* dW2, void* ws, size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X || !Wg || !W1 || !W2 || !dX_out || !saved || !dX || !dWg || !dW1 || !dW2 || !ws) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(W1, 16) || misaligned(W2, 16) || misaligned(dX_out, 16) ||
+      misaligned(dX, 16) || misaligned(dWg, 16) || misaligned(dW1, 16) || misaligned(dW2, 16) ||
+      misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D);
+  if (ws_bytes < W.total || saved_bytes < L.total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const char* sv = (const char*)saved; char* w = (char*)ws;
+  const float* S = (const float*)(sv + L.S); const int32_t* I = (const int32_t*)(sv + L.I);
+  const float* G = (const float*)(sv + L.G);
+  const int32_t* row_ptr = (const int32_t*)(sv + L.row_ptr); const int32_t* slots = (const int32_t*)(sv + L.slots);
+  const void* X_in = sv + L.X_in; const void* Z = sv + L.Z; const void* H = sv + L.H; const void* X_e = sv + L.X_e;
+  void* dX_e = w + W.dX_e; float* dG = (float*)(w + W.dG); void* dZ = w + W.dZ; void* dX_in = w + W.dX_in;
+  float* dL = (float*)(w + W.dL); float* part = (float*)(w + W.dWg_part);
+  int* status = (int*)(w + W.status);
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
+  // Eq. 4 backward: dX_e, dG
+  EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
+  // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
+  BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z};
+  if ((s = run_gemm(D, g3, status, st)) != EC_OK) return s;
+  // dW2[i] = dX_e[i]^T . H[i]
+  BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
+  if ((s = run_gemm(D, g4, status, st)) != EC_OK) return s;
+  // dW1[i] = X_in[i]^T . dZ[i]
+  BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
+  if ((s = run_gemm(D, g5, status, st)) != EC_OK) return s;
+  // dX_in[i] = dZ[i] . W1[i]^T
+  BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
+  if ((s = run_gemm(D, g6, status, st)) != EC_OK) return s;
+  // softmax backward: dL [n, E] fp32
+  EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, D.n, D.E, D.k, st));
+  // dWg = X^T . dL, split over the tokens into fixed chunks and summed in a fixed order
+  {
+    const int P = dwg_splits(D);
+    const int64_t chunk = (D.n + P - 1) / P;
+    GemmArgs g; memset(&g, 0, sizeof(g));
+    g.A = X; g.B = dL; g.C = part; g.a_dtype = D.dtype; g.b_dtype = EC_F32; g.c_dtype = EC_F32;
+    g.M = D.d; g.N = D.E; g.K = (int)chunk; g.batches = P; g.k_limit = D.n;
+    g.sam = 1; g.sak = D.d; g.sbk = D.E; g.sbn = 1; g.ldc = D.E;
+    g.batch_a = chunk * D.d; g.batch_b = chunk * D.E; g.batch_c = (int64_t)D.d * D.E;
+    g.epi = EPI_STORE;
+    EC_CUDA(launch_gemm_simt(g, st));
+    EC_CUDA(launch_reduce_partials(D.dtype, part, dWg, P, (int64_t)D.d * D.E, st));
+  }
+  // dX = dL . Wg^T + sum over the slots of each token of dX_in
+  {
+    GemmArgs g; memset(&g, 0, sizeof(g));
+    g.A = dL; g.B = Wg; g.C = dX; g.a_dtype = EC_F32; g.b_dtype = D.dtype; g.c_dtype = D.dtype;
+    g.M = (int)D.n; g.N = D.d; g.K = D.E; g.batches = 1;
+    g.sam = D.E; g.sak = 1; g.sbk = 1; g.sbn = D.E; g.ldc = D.d;
+    g.epi = EPI_ADD_SLOTS; g.row_ptr = row_ptr; g.slots = slots; g.rows = dX_in; g.ld_rows = D.d;
+    EC_CUDA(launch_gemm_simt(g, st));
+  }
+  return EC_OK;
+}
+
+ec_status ec_read_status(const void* ws, void* stream) {
+  if (!ws) return EC_ERR_INVALID_ARG;
+  StatusWord h;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return EC_ERR_CUDA;
+  if (cudaMemcpy(&h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return EC_ERR_CUDA;
+  return h.code == 0 ? EC_OK : (h.code == EC_ERR_TIMEOUT ? EC_ERR_TIMEOUT : EC_ERR_CUDA);
+}
+
+const char* ec_status_string(ec_status s) {
+  switch (s) {
+    case EC_OK: return "ok";
+    case EC_ERR_INVALID_ARG: return "invalid argument";
+    case EC_ERR_UNSUPPORTED: return "unsupported configuration";
+    case EC_ERR_WORKSPACE: return "workspace or saved buffer too small";
+    case EC_ERR_CUDA: return "CUDA call failed";
+    case EC_ERR_TIMEOUT: return "a bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+int ec_uses_tensor_cores(const ec_config* c) {
+  Dims D; if (check_cfg(c, &D) != EC_OK || D.dtype != EC_BF16) return 0;
+  TcGemmArgs t; memset(&t, 0, sizeof(t));
+  t.a_mn_major = 0; t.b_mn_major = 1; t.M = (int)D.k; t.N = D.dff; t.K = D.d; t.batches = D.E;
+  t.lda = D.d; t.ldb = D.dff; t.ldc = D.dff; t.epi = EPI_GELU;
+  t.A = t.B = t.C = (void*)16;   // shape query only
+  return tc_gemm_supported(t) ? 1 : 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of libecmoe.
+// Launch wrappers queue work on the given stream and return the launch status.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace ecmoe {
+
+using bf16 = __nv_bfloat16;
+
+constexpr int kTopkChunk = 32;     // experts per histogram CTA column chunk
+constexpr int kRadixPasses = 8;    // 8-bit digits of the 64-bit (score, token) key
+constexpr int kSortTile = 4096;    // 64-bit keys sorted in shared memory by one CTA
+
+// Word 0 of the workspace: status written by kernels (0 = fine, 5 = a bounded wait expired).
+struct StatusWord { int code; int where; int pad[62]; };
+
+// Per-expert state of the radix selection.
+struct SelState { unsigned long long prefix; unsigned int k_rem; unsigned int done; };
+
+// ---- routing (routing.cu) -------------------------------------------------------------------
+cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, float* S, int64_t n,
+                                     int d, int E, cudaStream_t st);
+// scratch layout for the selection is described in routing.cu; bytes needed:
+size_t topk_scratch_bytes(int64_t n, int E, int64_t k);
+cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I, float* G,
+                        void* scratch, cudaStream_t st);
+size_t inverse_scratch_bytes(int64_t n);
+cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t slots_total, int32_t* row_ptr,
+                                 int32_t* slots, void* scratch, cudaStream_t st);
+cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t slots_total,
+                          int d, cudaStream_t st);
+cudaError_t launch_combine(int dtype, const void* X_e, const float* G, const int32_t* row_ptr,
+                           const int32_t* slots, void* X_out, int64_t n, int d, cudaStream_t st);
+// dX_e[s,:] = G[s] * dX_out[I[s],:],  dG[s] = <dX_out[I[s],:], X_e[s,:]>
+cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const void* X_e, const float* G,
+                               const int32_t* I, void* dX_e, float* dG, int64_t slots_total, int d,
+                               cudaStream_t st);
+// dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] S[t,i']),  dS scattered from dG through the inverse index
+cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr,
+                               const int32_t* slots, float* dL, int64_t n, int E, int64_t k,
+                               cudaStream_t st);
+// out[r,c] = sum_p part[p,r,c] in ascending p (fixed order), cast to dtype
+cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems,
+                                   cudaStream_t st);
+
+// ---- plain FMA GEMM (gemm_simt.cu) -------------------------------------------------------------
+enum Epilogue { EPI_STORE = 0, EPI_GELU = 1, EPI_GELU_GRAD = 2, EPI_ADD_SLOTS = 3 };
+
+struct GemmArgs {
+  const void* A; const void* B; void* C;
+  int a_dtype, b_dtype, c_dtype;       // ec_dtype values; accumulation is always fp32
+  int M, N, K, batches;
+  int64_t sam, sak, sbk, sbn, ldc;     // element strides: A[m*sam + k*sak], B[k*sbk + n*sbn], C[m*ldc + n]
+  int64_t batch_a, batch_b, batch_c;   // element strides between batches
+  int64_t k_limit;                     // if > 0, batch b contracts only min(K, k_limit - b*K) terms (split of a long K)
+  int epi, gelu;
+  void* C2;                            // EPI_GELU: receives GeLU(acc) (C receives acc)
+  const void* Zin;                     // EPI_GELU_GRAD: C = acc * GeLU'(Zin), same layout and dtype as C
+  const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;  // EPI_ADD_SLOTS
+};
+cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
+
+// ---- tcgen05 GEMM (gemm_tc.cu) ---------------------------------------------------------------------
+struct TcGemmArgs {
+  // C[b][m][n] = sum_k A[b](m,k) * B[b](k,n), bf16 operands, fp32 accumulation in tensor memory.
+  const void* A; const void* B;
+  int a_mn_major;   // 0: A stored [batch][M][K] (K contiguous); 1: stored [batch][K][M]
+  int b_mn_major;   // 0: B stored [batch][N][K] (K contiguous); 1: stored [batch][K][N]
+  int M, N, K, batches;
+  int64_t lda, ldb; // elements between consecutive rows of the stored matrices
+  int64_t batch_a, batch_b;
+  int epi, gelu;    // EPI_STORE / EPI_GELU / EPI_GELU_GRAD, or EPI_SOFTMAX below
+  void* C; void* C2; const void* Zin; int64_t ldc; int64_t batch_c;   // bf16 outputs
+  float* S;         // EPI_SOFTMAX: fp32 row softmax of the N columns, [M, N]
+  int* status;      // device status word
+};
+constexpr int EPI_SOFTMAX = 4;
+bool tc_gemm_supported(const TcGemmArgs& g);
+cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st);
+
+}  // namespace ecmoe

@@ -1,0 +1,589 @@
+// Routing, shuffle and unshuffle kernels of the expert-choice layer (Section 3.2, Eq. 2-4)
+// and the element-wise parts of its backward pass.  Everything here is bandwidth- or
+// latency-bound integer / fp32 work; the dense contractions live in gemm_*.cu.
+#include "internal.h"
+
+namespace ecmoe {
+
+// ------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float ld_f(const float* p, int64_t i) { return p[i]; }
+__device__ __forceinline__ float ld_f(const bf16* p, int64_t i) { return __bfloat162float(p[i]); }
+
+template <typename T> struct Vec;            // one 16-byte vector of T
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  __device__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static uint4 pack(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                      __float_as_uint(f[3]));
+  }
+};
+template <> struct Vec<bf16> {
+  static constexpr int N = 8;
+  __device__ static void unpack(const uint4& v, float* f) {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {            // bf16 -> fp32 is a 16-bit shift
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  __device__ static uint4 pack(const float* f) {
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<unsigned*>(&p);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+static inline unsigned grid_for(int64_t work, int threads, int64_t cap = 148 * 16) {
+  int64_t b = (work + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > cap) b = cap;
+  return (unsigned)b;
+}
+
+// ------------------------------------------------------------------------------------------
+// Gate, Eq. 2: S = Softmax(X . Wg) over the experts of each token.  FMA version (fp32 path and
+// shapes the tensor-core kernel does not take).  One CTA handles TT tokens; the logits of the
+// TT x E (token, expert) pairs are spread over the threads.
+// ------------------------------------------------------------------------------------------
+constexpr int kGateTT = 8, kGateDC = 512, kGateThreads = 256, kGateMaxE = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kGateThreads)
+gate_softmax_simt_kernel(const T* __restrict__ X, const T* __restrict__ Wg, float* __restrict__ S,
+                         int64_t n, int d, int E) {
+  __shared__ float Xs[kGateTT][kGateDC];
+  __shared__ float Ls[kGateTT][kGateMaxE];
+  const int64_t t0 = (int64_t)blockIdx.x * kGateTT;
+  const int tid = threadIdx.x;
+  constexpr int R = kGateTT * kGateMaxE / kGateThreads;
+  float acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = 0.f;
+  const int pairs = kGateTT * E;
+  for (int d0 = 0; d0 < d; d0 += kGateDC) {
+    const int dc = min(kGateDC, d - d0);
+    for (int idx = tid; idx < kGateTT * dc; idx += kGateThreads) {
+      const int tt = idx / dc, dd = idx % dc;
+      const int64_t t = t0 + tt;
+      Xs[tt][dd] = t < n ? ld_f(X, t * d + d0 + dd) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int p = tid + r * kGateThreads;
+      if (p < pairs) {
+        const int tt = p / E, i = p % E;
+        float a = acc[r];
+        for (int dd = 0; dd < dc; ++dd) a = fmaf(Xs[tt][dd], ld_f(Wg, (int64_t)(d0 + dd) * E + i), a);
+        acc[r] = a;
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    const int p = tid + r * kGateThreads;
+    if (p < pairs) Ls[p / E][p % E] = acc[r];
+  }
+  __syncthreads();
+  const int warp = tid >> 5, lane = tid & 31;     // one warp per token
+  const int64_t t = t0 + warp;
+  if (warp < kGateTT && t < n) {
+    float mx = -INFINITY;
+    for (int i = lane; i < E; i += 32) mx = fmaxf(mx, Ls[warp][i]);
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+    for (int i = lane; i < E; i += 32) { const float e = expf(Ls[warp][i] - mx); Ls[warp][i] = e; sum += e; }
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float inv = 1.f / sum;
+    for (int i = lane; i < E; i += 32) S[t * E + i] = Ls[warp][i] * inv;
+  }
+}
+
+cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, float* S, int64_t n,
+                                     int d, int E, cudaStream_t st) {
+  const unsigned grid = (unsigned)((n + kGateTT - 1) / kGateTT);
+  if (dtype == 0)
+    gate_softmax_simt_kernel<float><<<grid, kGateThreads, 0, st>>>((const float*)X, (const float*)Wg, S, n, d, E);
+  else
+    gate_softmax_simt_kernel<bf16><<<grid, kGateThreads, 0, st>>>((const bf16*)X, (const bf16*)Wg, S, n, d, E);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Column top-k, Eq. 2: G, I = TopK(S^T, k).
+//
+// Every (token t, expert i) entry gets the 64-bit key  (~bits(S[t,i]) << 32) | t.  S >= 0, so its
+// bit pattern is monotone in its value: a smaller key is a larger score, and among equal scores a
+// lower token.  Keys of one expert are distinct, so "the k smallest keys, ascending" is the
+// unique answer with ties broken toward the lower token and slots listed by descending score.
+//
+// Selection is a most-significant-digit radix select run for all experts at once: pass p
+// histograms digit p (8 bits) of the keys that still match the expert's prefix; the last CTA of a
+// column chunk to finish picks the digit in which the k-th key lies.  An expert is finished as
+// soon as the bucket it descends into holds exactly the number of keys still wanted (with
+// distinct scores that is after the four score digits; the token digits only run for ties at
+// the threshold).  Then one pass copies the keys not above the threshold and a bitonic network
+// sorts the k keys of each expert.
+//
+// scratch: [SelState E][hist passes*E*256 u32][counters passes*chunks u32][cursor E u32][keys E*kpad u64]
+// ------------------------------------------------------------------------------------------
+constexpr int kHistThreads = 256;
+
+__device__ __forceinline__ unsigned long long make_key(float s, int64_t t) {
+  return ((unsigned long long)(~__float_as_uint(s)) << 32) | (unsigned long long)(unsigned)t;
+}
+
+struct TopkLayout {
+  size_t off_state, off_hist, off_counters, off_cursor, off_keys, zero_bytes, total;
+  int chunks; int64_t kpad;
+};
+static TopkLayout topk_layout(int64_t n, int E, int64_t k) {
+  TopkLayout L;
+  L.chunks = (E + kTopkChunk - 1) / kTopkChunk;
+  L.kpad = 1; while (L.kpad < k) L.kpad <<= 1;
+  size_t o = 0;
+  auto take = [&](size_t b) { size_t r = o; o += (b + 255) & ~(size_t)255; return r; };
+  L.off_state = take(sizeof(SelState) * (size_t)E);
+  L.off_hist = take((size_t)kRadixPasses * E * 256 * 4);
+  L.off_counters = take((size_t)kRadixPasses * L.chunks * 4);
+  L.off_cursor = take((size_t)E * 4);
+  L.zero_bytes = o;                       // everything up to here starts at zero
+  L.off_keys = take((size_t)E * L.kpad * 8);
+  L.total = o;
+  return L;
+}
+size_t topk_scratch_bytes(int64_t n, int E, int64_t k) { return topk_layout(n, E, k).total; }
+
+// maps the lanes of a warp on a [rows x cw] slab of S: cwp = power of two >= cw
+__device__ __forceinline__ int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+
+__global__ void __launch_bounds__(kHistThreads)
+topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int pass, int rows_per_cta,
+                 SelState* state, unsigned* hist, unsigned* counters) {
+  __shared__ unsigned sh[256 * kTopkChunk];            // [digit][column]
+  __shared__ unsigned long long s_prefix[kTopkChunk];
+  __shared__ int s_active[kTopkChunk];
+  __shared__ int s_any, s_last;
+  const int tid = threadIdx.x, chunk = blockIdx.y, nchunks = gridDim.y;
+  const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
+  if (tid == 0) s_any = 0;
+  __syncthreads();
+  if (tid < kTopkChunk) {
+    int act = 0; unsigned long long pre = 0;
+    if (tid < cw) {
+      if (pass == 0) act = 1;
+      else { act = state[c0 + tid].done ? 0 : 1; pre = state[c0 + tid].prefix; }
+    }
+    s_active[tid] = act; s_prefix[tid] = pre;
+    if (act) s_any = 1;
+  }
+  for (int i = tid; i < 256 * kTopkChunk; i += kHistThreads) sh[i] = 0;
+  __syncthreads();
+  if (!s_any) return;                                  // uniform: every expert of the chunk is finished
+  const int shift = 56 - 8 * pass;
+  const int cwp = pow2_at_least(cw), rpw = 32 / cwp;
+  const int warp = tid >> 5, lane = tid & 31, nwarps = kHistThreads / 32;
+  const int r = lane / cwp, cc = lane % cwp;
+  const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
+  const int64_t t1 = min(n, t0 + rows_per_cta);
+  if (cc < cw && s_active[cc]) {
+    const unsigned long long pre = s_prefix[cc];
+    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw) {
+      const unsigned long long key = make_key(S[t * E + c0 + cc], t);
+      const bool match = pass == 0 || ((key ^ pre) >> (shift + 8)) == 0;
+      if (match) atomicAdd(&sh[(unsigned)((key >> shift) & 255) * kTopkChunk + cc], 1u);
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < 256 * kTopkChunk; i += kHistThreads) {
+    const unsigned v = sh[i];
+    const int col = i % kTopkChunk, dig = i / kTopkChunk;
+    if (v) atomicAdd(&hist[((size_t)pass * E + c0 + col) * 256 + dig], v);
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&counters[pass * nchunks + chunk], 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // The last CTA of this chunk sees the full histograms: descend one digit per active expert.
+  for (int col = warp; col < cw; col += nwarps) {
+    if (!s_active[col]) continue;
+    const unsigned* h = hist + ((size_t)pass * E + c0 + col) * 256;
+    unsigned cnt[8], lsum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { cnt[j] = __ldcg(h + lane * 8 + j); lsum += cnt[j]; }
+    unsigned incl = lsum;
+    for (int o = 1; o < 32; o <<= 1) { const unsigned v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+    const unsigned excl = incl - lsum;
+    const unsigned k_rem = pass == 0 ? k : state[c0 + col].k_rem;
+    if (excl < k_rem && k_rem <= incl) {               // exactly one lane
+      unsigned before = excl; int D = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (before < k_rem && k_rem <= before + cnt[j]) { D = j; break; }
+        before += cnt[j];
+      }
+      const unsigned in_bucket = cnt[D];
+      const unsigned new_rem = k_rem - before;
+      unsigned long long pre = s_prefix[col] | ((unsigned long long)(lane * 8 + D) << shift);
+      SelState ns;
+      ns.k_rem = new_rem;
+      ns.done = (in_bucket == new_rem) ? 1u : 0u;
+      if (ns.done && shift > 0) pre |= (1ull << shift) - 1ull;   // whole bucket is taken
+      ns.prefix = pre;
+      state[c0 + col] = ns;
+    }
+  }
+}
+
+// Copies the keys not above each expert's threshold to keys[i][0..k), in no particular order.
+__global__ void __launch_bounds__(kHistThreads)
+topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int64_t kpad,
+                    int rows_per_cta, const SelState* __restrict__ state, unsigned* cursor,
+                    unsigned long long* keys) {
+  __shared__ unsigned s_cnt[kTopkChunk], s_base[kTopkChunk];
+  __shared__ unsigned long long s_thr[kTopkChunk];
+  const int tid = threadIdx.x, chunk = blockIdx.y;
+  const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
+  if (tid < kTopkChunk) { s_cnt[tid] = 0; s_thr[tid] = tid < cw ? state[c0 + tid].prefix : 0ull; }
+  __syncthreads();
+  const int cwp = pow2_at_least(cw), rpw = 32 / cwp;
+  const int warp = tid >> 5, lane = tid & 31, nwarps = kHistThreads / 32;
+  const int r = lane / cwp, cc = lane % cwp;
+  const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
+  const int64_t t1 = min(n, t0 + rows_per_cta);
+  unsigned long long thr = 0;
+  if (cc < cw) {
+    thr = s_thr[cc];
+    unsigned mine = 0;
+    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw)
+      mine += make_key(S[t * E + c0 + cc], t) <= thr ? 1u : 0u;
+    if (mine) atomicAdd(&s_cnt[cc], mine);
+  }
+  __syncthreads();
+  if (tid < cw) { const unsigned c = s_cnt[tid]; s_base[tid] = c ? atomicAdd(&cursor[c0 + tid], c) : 0u; }
+  __syncthreads();
+  if (tid < kTopkChunk) s_cnt[tid] = 0;
+  __syncthreads();
+  if (cc < cw) {
+    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw) {
+      const unsigned long long key = make_key(S[t * E + c0 + cc], t);
+      if (key <= thr) {
+        const unsigned pos = s_base[cc] + atomicAdd(&s_cnt[cc], 1u);
+        if (pos < k) keys[(size_t)(c0 + cc) * kpad + pos] = key;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, float* G, int64_t o) {
+  I[o] = (int32_t)(unsigned)(key & 0xFFFFFFFFull);
+  G[o] = __uint_as_float(~(unsigned)(key >> 32));
+}
+
+// Bitonic steps on one tile of kSortTile keys held in shared memory.  Runs the network sizes
+// size_lo..size_hi (powers of two); for a size larger than the tile only the strides that fit.
+constexpr int kSortThreads = 1024;
+__global__ void __launch_bounds__(kSortThreads)
+topk_sort_tile_kernel(unsigned long long* keys, int64_t kpad, int64_t k, int64_t size_lo, int64_t size_hi,
+                      int emit, int32_t* I, float* G) {
+  __shared__ unsigned long long sk[kSortTile];
+  const int64_t tiles_per_expert = (kpad + kSortTile - 1) / kSortTile;
+  const int64_t expert = blockIdx.x / tiles_per_expert;
+  const int64_t base = (blockIdx.x % tiles_per_expert) * kSortTile;   // index inside the expert
+  const int len = (int)min((int64_t)kSortTile, kpad - base);          // power of two
+  unsigned long long* src = keys + expert * kpad + base;
+  for (int i = threadIdx.x; i < len; i += kSortThreads) sk[i] = src[i];
+  __syncthreads();
+  for (int64_t size = size_lo; size <= size_hi; size <<= 1) {
+    for (int64_t stride = min(size >> 1, (int64_t)(len >> 1)); stride >= 1; stride >>= 1) {
+      for (int p = threadIdx.x; p < (len >> 1); p += kSortThreads) {
+        const int i = (int)((p / stride) * 2 * stride + (p % stride));
+        const int j = i + (int)stride;
+        const bool asc = ((base + i) & size) == 0;
+        const unsigned long long a = sk[i], b = sk[j];
+        if ((a > b) == asc) { sk[i] = b; sk[j] = a; }
+      }
+      __syncthreads();
+    }
+  }
+  if (emit) {
+    for (int i = threadIdx.x; i < len; i += kSortThreads)
+      if (base + i < k) emit_slot(sk[i], I, G, expert * k + base + i);
+  } else {
+    for (int i = threadIdx.x; i < len; i += kSortThreads) src[i] = sk[i];
+  }
+}
+
+// One compare-exchange step at a stride that spans tiles.
+__global__ void topk_sort_global_kernel(unsigned long long* keys, int64_t kpad, int64_t total_pairs,
+                                        int64_t size, int64_t stride) {
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < total_pairs;
+       p += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t expert = p / (kpad >> 1), q = p % (kpad >> 1);
+    const int64_t i = (q / stride) * 2 * stride + (q % stride), j = i + stride;
+    unsigned long long* kk = keys + expert * kpad;
+    const bool asc = (i & size) == 0;
+    const unsigned long long a = kk[i], b = kk[j];
+    if ((a > b) == asc) { kk[i] = b; kk[j] = a; }
+  }
+}
+
+cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I, float* G,
+                        void* scratch, cudaStream_t st) {
+  const TopkLayout L = topk_layout(n, E, k);
+  char* base = (char*)scratch;
+  SelState* state = (SelState*)(base + L.off_state);
+  unsigned* hist = (unsigned*)(base + L.off_hist);
+  unsigned* counters = (unsigned*)(base + L.off_counters);
+  unsigned* cursor = (unsigned*)(base + L.off_cursor);
+  unsigned long long* keys = (unsigned long long*)(base + L.off_keys);
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(base, 0, L.zero_bytes, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(keys, 0xFF, (size_t)E * L.kpad * 8, st)) != cudaSuccess) return e;
+  // rows per CTA: enough CTAs to fill the machine a few times over, at least 64 rows each
+  int64_t want = (int64_t)148 * 8 / L.chunks; if (want < 1) want = 1;
+  int64_t rows = (n + want - 1) / want; if (rows < 64) rows = 64;
+  const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks);
+  for (int pass = 0; pass < kRadixPasses; ++pass)
+    topk_hist_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
+  topk_compact_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys);
+  const int64_t tiles = (L.kpad + kSortTile - 1) / kSortTile;
+  const unsigned sort_grid = (unsigned)(E * tiles);
+  if (L.kpad <= kSortTile) {
+    topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, L.kpad, 1, I, G);
+  } else {
+    topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, kSortTile, 0, I, G);
+    const int64_t pairs = (int64_t)E * (L.kpad >> 1);
+    for (int64_t size = 2 * kSortTile; size <= L.kpad; size <<= 1) {
+      for (int64_t stride = size >> 1; stride >= kSortTile; stride >>= 1)
+        topk_sort_global_kernel<<<grid_for(pairs, 256), 256, 0, st>>>(keys, L.kpad, pairs, size, stride);
+      topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, size, size, size == L.kpad, I, G);
+    }
+  }
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Index form of P = Onehot(I) (Eq. 2) read by token: row_ptr / slots.
+// Integer atomics only count and hand out positions; each token's short list is then sorted,
+// so the result does not depend on the order in which threads ran.
+// scratch: [cursor n int32]
+// ------------------------------------------------------------------------------------------
+size_t inverse_scratch_bytes(int64_t n) { return ((size_t)(n + 1) * 4 + 255) & ~(size_t)255; }
+
+__global__ void inv_count_kernel(const int32_t* __restrict__ I, int64_t total, int32_t* cnt) {
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x)
+    atomicAdd(&cnt[I[s]], 1);
+}
+
+// exclusive scan of cnt[0..n) into row_ptr[0..n], single CTA
+__global__ void __launch_bounds__(1024) inv_scan_kernel(const int32_t* __restrict__ cnt, int64_t n, int32_t* row_ptr) {
+  __shared__ int s_sum[1024];
+  const int tid = threadIdx.x;
+  const int64_t per = (n + 1023) / 1024;
+  const int64_t a = min(n, tid * per), b = min(n, a + per);
+  int sum = 0;
+  for (int64_t t = a; t < b; ++t) sum += cnt[t];
+  s_sum[tid] = sum;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {
+    const int v = tid >= o ? s_sum[tid - o] : 0;
+    __syncthreads();
+    s_sum[tid] += v;
+    __syncthreads();
+  }
+  int run = s_sum[tid] - sum;
+  for (int64_t t = a; t < b; ++t) { row_ptr[t] = run; run += cnt[t]; }
+  if (tid == 1023) row_ptr[n] = s_sum[1023];
+}
+
+__global__ void inv_fill_kernel(const int32_t* __restrict__ I, int64_t total, const int32_t* __restrict__ row_ptr,
+                                int32_t* cursor, int32_t* slots) {
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
+    const int t = I[s];
+    slots[row_ptr[t] + atomicAdd(&cursor[t], 1)] = (int32_t)s;
+  }
+}
+
+__global__ void inv_sort_kernel(const int32_t* __restrict__ row_ptr, int64_t n, int32_t* slots) {
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += (int64_t)gridDim.x * blockDim.x) {
+    const int a = row_ptr[t], b = row_ptr[t + 1];
+    for (int i = a + 1; i < b; ++i) {
+      const int v = slots[i]; int j = i - 1;
+      while (j >= a && slots[j] > v) { slots[j + 1] = slots[j]; --j; }
+      slots[j + 1] = v;
+    }
+  }
+}
+
+cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int32_t* row_ptr, int32_t* slots,
+                                 void* scratch, cudaStream_t st) {
+  int32_t* cursor = (int32_t*)scratch;
+  cudaError_t e;
+  // counts are built in slots' neighbour: reuse row_ptr[1..n] would break the scan, so count in `cursor`
+  if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cursor);
+  inv_scan_kernel<<<1, 1024, 0, st>>>(cursor, n, row_ptr);
+  if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cursor, slots);
+  inv_sort_kernel<<<grid_for(n, 256), 256, 0, st>>>(row_ptr, n, slots);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Shuffle, Eq. 3: X_in = P . X as an indexed row copy in 16-byte vectors.
+// ------------------------------------------------------------------------------------------
+__global__ void gather_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ I, uint4* __restrict__ X_in,
+                              int64_t total_vec, int vec_per_row) {
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_vec; g += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t s = g / vec_per_row; const int v = (int)(g % vec_per_row);
+    X_in[g] = X[(int64_t)I[s] * vec_per_row + v];
+  }
+}
+
+cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t total, int d, cudaStream_t st) {
+  const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
+  const int64_t tv = total * vpr;
+  gather_kernel<<<grid_for(tv, 256, 148 * 32), 256, 0, st>>>((const uint4*)X, I, (uint4*)X_in, tv, vpr);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Unshuffle, Eq. 4: X_out[t,:] = sum over the slots of t (ascending expert) of G[s] * X_e[s,:].
+// Read through the token->slot index, so no atomics and a fixed summation order.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void combine_kernel(const uint4* __restrict__ X_e, const float* __restrict__ G,
+                               const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
+                               uint4* __restrict__ X_out, int64_t total_vec, int vec_per_row) {
+  constexpr int N = Vec<T>::N;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_vec; g += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = g / vec_per_row; const int v = (int)(g % vec_per_row);
+    float acc[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc[i] = 0.f;
+    const int a = row_ptr[t], b = row_ptr[t + 1];
+    for (int q = a; q < b; ++q) {
+      const int s = slots[q];
+      const float w = G[s];
+      float x[N];
+      Vec<T>::unpack(X_e[(int64_t)s * vec_per_row + v], x);
+#pragma unroll
+      for (int i = 0; i < N; ++i) acc[i] = fmaf(w, x[i], acc[i]);
+    }
+    X_out[g] = Vec<T>::pack(acc);
+  }
+}
+
+cudaError_t launch_combine(int dtype, const void* X_e, const float* G, const int32_t* row_ptr, const int32_t* slots,
+                           void* X_out, int64_t n, int d, cudaStream_t st) {
+  const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
+  const int64_t tv = n * vpr;
+  const unsigned grid = grid_for(tv, 256, 148 * 32);
+  if (dtype == 0) combine_kernel<float><<<grid, 256, 0, st>>>((const uint4*)X_e, G, row_ptr, slots, (uint4*)X_out, tv, vpr);
+  else combine_kernel<bf16><<<grid, 256, 0, st>>>((const uint4*)X_e, G, row_ptr, slots, (uint4*)X_out, tv, vpr);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Backward of Eq. 4 per slot s = (i, j) holding token t:
+//   dX_e[s,:] = G[s] * dX_out[t,:],   dG[s] = <dX_out[t,:], X_e[s,:]>.   One warp per slot.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void bwd_combine_kernel(const uint4* __restrict__ dX_out, const uint4* __restrict__ X_e,
+                                   const float* __restrict__ G, const int32_t* __restrict__ I,
+                                   uint4* __restrict__ dX_e, float* __restrict__ dG, int64_t total, int vec_per_row) {
+  constexpr int N = Vec<T>::N;
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t s = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; s < total; s += warps) {
+    const int64_t t = I[s];
+    const float w = G[s];
+    float dot = 0.f;
+    for (int v = lane; v < vec_per_row; v += 32) {
+      float dy[N], xe[N], o[N];
+      Vec<T>::unpack(dX_out[t * vec_per_row + v], dy);
+      Vec<T>::unpack(X_e[s * vec_per_row + v], xe);
+#pragma unroll
+      for (int i = 0; i < N; ++i) { o[i] = w * dy[i]; dot = fmaf(dy[i], xe[i], dot); }
+      dX_e[s * vec_per_row + v] = Vec<T>::pack(o);
+    }
+    for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (lane == 0) dG[s] = dot;
+  }
+}
+
+cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const void* X_e, const float* G, const int32_t* I,
+                               void* dX_e, float* dG, int64_t total, int d, cudaStream_t st) {
+  const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
+  const unsigned grid = grid_for(total * 32, 256, 148 * 16);
+  if (dtype == 0) bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const uint4*)dX_out, (const uint4*)X_e, G, I, (uint4*)dX_e, dG, total, vpr);
+  else bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const uint4*)dX_out, (const uint4*)X_e, G, I, (uint4*)dX_e, dG, total, vpr);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Backward of the softmax of Eq. 2, one warp per token.  dS[t,i] is dG of the slot of expert i that
+// holds t (0 if none);  dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] * S[t,i']).
+// ------------------------------------------------------------------------------------------
+__global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __restrict__ dG,
+                                   const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
+                                   float* __restrict__ dL, int64_t n, int E, int64_t k) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < n; t += warps) {
+    const int a = row_ptr[t], b = row_ptr[t + 1];
+    float dot = 0.f;
+    for (int q = a + lane; q < b; q += 32) {
+      const int s = slots[q];
+      dot = fmaf(dG[s], S[t * E + s / k], dot);
+    }
+    for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    for (int i = lane; i < E; i += 32) dL[t * E + i] = -S[t * E + i] * dot;
+    __syncwarp();
+    for (int q = a + lane; q < b; q += 32) {           // the slots of one token belong to distinct experts
+      const int s = slots[q]; const int64_t i = s / k;
+      dL[t * E + i] = S[t * E + i] * (dG[s] - dot);
+    }
+  }
+}
+
+cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr, const int32_t* slots,
+                               float* dL, int64_t n, int E, int64_t k, cudaStream_t st) {
+  bwd_softmax_kernel<<<grid_for(n * 32, 256, 148 * 16), 256, 0, st>>>(S, dG, row_ptr, slots, dL, n, E, k);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Fixed-order sum of split partial results.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void reduce_partials_kernel(const float* __restrict__ part, T* __restrict__ out, int P, int64_t elems) {
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < elems; g += (int64_t)gridDim.x * blockDim.x) {
+    float acc = 0.f;
+    for (int p = 0; p < P; ++p) acc += part[(int64_t)p * elems + g];
+    if constexpr (sizeof(T) == 4) out[g] = acc; else out[g] = __float2bfloat16(acc);
+  }
+}
+
+cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems, cudaStream_t st) {
+  if (dtype == 0) reduce_partials_kernel<float><<<grid_for(elems, 256), 256, 0, st>>>(part, (float*)out, P, elems);
+  else reduce_partials_kernel<bf16><<<grid_for(elems, 256), 256, 0, st>>>(part, (bf16*)out, P, elems);
+  return cudaGetLastError();
+}
+
+}  // namespace ecmoe

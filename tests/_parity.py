@@ -1,0 +1,79 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI and
+compare it with the CPU oracle following the protocol
+
+  (i)   S_gpu against the oracle's own S, by tolerance;
+  (ii)  routing: the oracle's top-k and inverse index evaluated ON S_gpu must equal
+        I, G, row_ptr, slots from the GPU bit for bit;
+  (iii) every later tensor against the oracle evaluated with S and I fixed to the
+        GPU's (a one-ulp difference in S may legitimately flip a boundary token).
+
+Error measure: max|gpu - ref| / RMS(ref), per tensor.
+"""
+import numpy as np
+import torch
+
+from oracle import ec_oracle as O
+from paper_2202_09368_b200 import binding as B
+
+TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}
+
+
+def rel_err(got, ref):
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    rms = np.sqrt(np.mean(ref * ref))
+    if rms == 0:
+        return float(np.max(np.abs(got)))
+    return float(np.max(np.abs(got - ref)) / rms)
+
+
+def to_np(t):
+    return t.detach().float().cpu().numpy().astype(np.float64) if t.is_floating_point() else t.cpu().numpy()
+
+
+def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
+    """Step (ii): bit-exact routing given the GPU's own S."""
+    k = B.ec_capacity(cfg)
+    S32 = S_gpu.cpu().numpy()                      # float32 bits, compared as such
+    G_ref, I_ref = O.topk(S32, k)
+    I_np = I_gpu.cpu().numpy()
+    assert np.array_equal(I_np, I_ref), f"I differs in {(I_np != I_ref).sum()} of {I_ref.size} slots"
+    assert np.array_equal(G_gpu.cpu().numpy().view(np.uint32), G_ref.view(np.uint32))
+    rp_ref, sl_ref = O.inverse_index(I_ref, cfg.n)
+    assert np.array_equal(row_ptr.cpu().numpy(), rp_ref)
+    assert np.array_equal(slots.cpu().numpy(), sl_ref)
+    return I_ref
+
+
+def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True):
+    """Runs forward (+ backward) on the GPU and checks every tensor against the oracle."""
+    tol = TOL[dtype]
+    cfg = B.make_config(n, d, dff, E, c, dtype, gelu)
+    dev = "cuda"
+    X, Wg, W1, W2 = (t.to(dev) for t in (li.X, li.Wg, li.W1, li.W2))
+    ws = B.alloc_workspace(cfg)
+    X_out, saved = B.ec_moe_forward(cfg, X, Wg, W1, W2, ws=ws)
+    assert B.ec_read_status(ws) == B.EC_OK
+    v = B.saved_view(cfg, saved)
+    Xn, Wgn, W1n, W2n = (to_np(t) for t in (li.X, li.Wg, li.W1, li.W2))
+    errs = {}
+    if check_S:
+        errs["S"] = rel_err(to_np(v["S"]), O.gate(Xn, Wgn))
+        assert errs["S"] <= tol, errs
+    check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
+    f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy())
+    assert np.array_equal(v["X_in"].float().cpu().numpy(), Xn[f["I"]].astype(np.float32))   # gather is a copy
+    for name in ("Z", "H", "X_e"):
+        errs[name] = rel_err(to_np(v[name]), f[name])
+    errs["X_out"] = rel_err(to_np(X_out), f["X_out"])
+    cnt = O.experts_per_token(f["row_ptr"])
+    assert torch.all(X_out[torch.from_numpy(cnt == 0).to(dev)] == 0)
+    if backward:
+        dY = li.dX_out.to(dev)
+        dX, dWg, dW1, dW2 = B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, ws=ws)
+        assert B.ec_read_status(ws) == B.EC_OK
+        b = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), f, gelu)
+        for name, t in (("dX", dX), ("dWg", dWg), ("dW1", dW1), ("dW2", dW2)):
+            errs[name] = rel_err(to_np(t), b[name])
+    bad = {k_: e for k_, e in errs.items() if not e <= tol}
+    assert not bad, f"over tolerance {tol}: {bad} (all: {errs})"
+    return errs

@@ -1,0 +1,112 @@
+"""CUDA path against the CPU oracle, through the C ABI.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ec_oracle as O
+from paper_2202_09368_b200 import binding as B
+from paper_2202_09368_b200 import inputs as IN
+
+from _parity import TOL, check_routing, rel_err, run_and_check, to_np
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = torch.float32, torch.bfloat16
+
+
+@pytest.mark.parametrize("n,d,dff,E,c", [
+    (256, 64, 256, 4, 2.0),        # the tiny configuration
+    (300, 36, 100, 3, 1.5),        # ragged everywhere: k = 150, tiles with tails
+    (64, 16, 32, 1, 1.0),          # one expert: dense FFN
+    (48, 8, 16, 4, 4.0),           # c = E: every expert takes every token
+    (130, 12, 20, 8, 0.5),         # some tokens unselected; k = 8
+    (97, 8, 8, 5, 0.06),           # k = 1
+])
+def test_fp32_forward_backward(n, d, dff, E, c):
+    li = IN.make_layer_inputs(n, d, dff, E, F32, seed=0)
+    run_and_check(n, d, dff, E, c, F32, li)
+
+
+def test_fp32_tanh_gelu():
+    li = IN.make_layer_inputs(128, 32, 64, 4, F32, seed=1)
+    run_and_check(128, 32, 64, 4, 2.0, F32, li, gelu="tanh")
+
+
+@pytest.mark.parametrize("n,d,dff,E,c", [
+    (256, 64, 256, 4, 2.0),
+    (512, 128, 384, 8, 2.0),       # k = 128: one full MMA tile per expert
+    (1000, 200, 328, 16, 2.0),     # k = 125, ragged in every dimension
+    (2048, 256, 512, 32, 2.0),
+    (384, 64, 128, 3, 1.0),        # E not a multiple of 8
+    (1024, 192, 448, 64, 0.5),     # k = 8
+])
+def test_bf16_forward_backward(n, d, dff, E, c):
+    li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=0)
+    run_and_check(n, d, dff, E, c, BF16, li)
+
+
+def test_bf16_logit_scale_and_tanh():
+    li = IN.make_layer_inputs(1024, 128, 256, 16, BF16, seed=2, logit_scale=4.0)
+    run_and_check(1024, 128, 256, 16, 1.0, BF16, li, gelu="tanh")
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("n,d,E,c,levels", [(512, 16, 4, 2.0, 2), (777, 8, 3, 1.0, 1), (4096, 64, 32, 2.0, 3)])
+def test_routing_with_heavy_ties(n, d, E, c, levels, dtype):
+    """Few distinct logits: columns of S are full of exact ties; the lower token must win."""
+    X, Wg = IN.quantised_gate_inputs(n, d, E, levels, dtype)
+    cfg = B.make_config(n, d, 16, E, c, dtype)
+    r = B.ec_route(cfg, X.cuda(), Wg.cuda())
+    assert len(np.unique(r.S.cpu().numpy()[:, 0])) <= 2 * levels + 1
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+def test_routing_all_equal_scores():
+    n, d, E = 1500, 8, 6
+    X = torch.zeros(n, d)
+    Wg = torch.zeros(d, E)
+    cfg = B.make_config(n, d, 16, E, 2.0, F32)
+    r = B.ec_route(cfg, X.cuda(), Wg.cuda())
+    k = B.ec_capacity(cfg)
+    assert torch.equal(r.I.cpu(), torch.arange(k, dtype=torch.int32).repeat(E, 1))
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+@pytest.mark.parametrize("n,E,c", [(20000, 2, 2.0), (70000, 8, 2.0), (5000, 200, 2.0), (33000, 40, 0.7)])
+def test_routing_large_k_and_many_experts(n, E, c):
+    """k beyond one sort tile (multi-kernel bitonic path) and E beyond one column chunk."""
+    d = 16
+    li = IN.make_layer_inputs(n, d, 8, E, F32, seed=3, with_grad=False)
+    cfg = B.make_config(n, d, 16, E, c, F32)
+    r = B.ec_route(cfg, li.X.cuda(), li.Wg.cuda())
+    assert rel_err(to_np(r.S), O.gate(to_np(li.X), to_np(li.Wg))) <= 1e-4
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+def test_run_to_run_determinism():
+    n, d, dff, E = 1024, 128, 256, 8
+    li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=5)
+    cfg = B.make_config(n, d, dff, E, 2.0, BF16)
+    X, Wg, W1, W2, dY = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2, li.dX_out))
+    outs = []
+    for _ in range(2):
+        Y, saved = B.ec_moe_forward(cfg, X, Wg, W1, W2)
+        g = B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved)
+        outs.append([Y.clone()] + [t.clone() for t in g] + [saved.clone()])
+    for a, b in zip(*outs):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    cfg = B.make_config(256, 64, 256, 4, 2.0, F32)
+    li = IN.make_layer_inputs(256, 64, 256, 4, F32)
+    X, Wg = li.X.cuda(), li.Wg.cuda()
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.EcError) as e:
+        B.ec_route(cfg, X, Wg, ws=small)
+    assert e.value.code == B.EC_ERR_WORKSPACE
+    ws = B.alloc_workspace(cfg)
+    with pytest.raises(B.EcError) as e:
+        B.ec_route(cfg, X.view(-1)[1:], Wg, ws=ws)          # misaligned pointer
+    assert e.value.code == B.EC_ERR_INVALID_ARG
+    torch.cuda.synchronize()
