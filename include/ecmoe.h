@@ -20,7 +20,7 @@
  *  - Errors are return codes.  Arguments are checked on the host before anything
  *    is launched; nothing is launched when the code is not EC_OK.
  *  - X, Wg, W1, W2, X_out, dX_out and all gradients have the element type
- *    cfg->dtype; S and G are always fp32 and index outputs are int32.
+ *    cfg->dtype; S, G and X_e are always fp32 and index outputs are int32.
  *  - Restrictions (EC_ERR_UNSUPPORTED otherwise): d_model and d_ff rows must be a
  *    multiple of 16 bytes long; n < 2^31; 1 <= E <= 256; E*k < 2^31; groups == 1.
  */
@@ -68,7 +68,7 @@ typedef struct {
   void* X_in;       /* [E, k, d]  gathered expert inputs (Eq. 3)                       */
   void* Z;          /* [E, k, d'] X_in[i] . W1[i]                                      */
   void* H;          /* [E, k, d'] GeLU(Z)                                              */
-  void* X_e;        /* [E, k, d]  expert outputs H[i] . W2[i]^T                        */
+  float* X_e;       /* [E, k, d]  expert outputs H[i] . W2[i]^T, fp32 on both paths    */
 } ec_saved_ptrs;
 
 /* Eq. 1: k = floor(n*c/E).  Returns -1 when cfg is NULL or k falls outside [1, n]. */

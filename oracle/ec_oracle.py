@@ -116,12 +116,22 @@ def route(X, Wg, c: float, S_override=None):
     return dict(k=k, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots)
 
 
-def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None):
+def _keep(name, x):
+    return x
+
+
+def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
+            store=_keep):
     """Eq. 1-4.  Returns every intermediate.
 
     S_override replaces the gate output (the routing is then taken from it);
     I_override additionally fixes the index matrix (G is read from S at I).
     Both exist so that later stages can be compared on identical routing.
+
+    `store(name, array)` is applied to each tensor at the point where the layer
+    keeps it in memory (Z, H, X_e, X_out).  The default keeps fp64, which is the
+    definition; a test passes a rounding function to measure how far a storage
+    format alone moves the result (the arithmetic floor of a low-precision path).
     """
     X = np.asarray(X, F64); Wg = np.asarray(Wg, F64)
     W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
@@ -137,19 +147,21 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
     I, G = r["I"], r["G"]
     X_in = X[I]                                            # Eq. 3: X_in = P . X,  [e, k, d]
     Z = np.stack([X_in[i] @ W1[i] for i in range(e)])      # [e, k, d']
-    H = gelu(Z, gelu_variant)
-    X_e = np.stack([H[i] @ W2[i].T for i in range(e)])     # [e, k, d]
+    H = store("H", gelu(Z, gelu_variant))
+    Z = store("Z", Z)
+    X_e = store("X_e", np.stack([H[i] @ W2[i].T for i in range(e)]))   # [e, k, d]
     X_out = np.zeros((n, d), F64)                          # Eq. 4, experts in ascending order
     for i in range(e):
         for j in range(k):
             X_out[I[i, j]] += G[i, j] * X_e[i, j]
+    X_out = store("X_out", X_out)
     r.update(X_in=X_in, Z=Z, H=H, X_e=X_e, X_out=X_out)
     return r
 
 
-def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf"):
+def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep):
     """Gradients of <dX_out, X_out> with respect to X, Wg, W1, W2 by the chain rule
-    through Eq. 4, 3, 2 in that order, with I held constant."""
+    through Eq. 4, 3, 2 in that order, with I held constant.  `store` as in forward()."""
     X = np.asarray(X, F64); Wg = np.asarray(Wg, F64)
     W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
     dX_out = np.asarray(dX_out, F64)
@@ -159,22 +171,23 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf"):
     X_in, Z, H, X_e = fwd["X_in"], fwd["Z"], fwd["H"], fwd["X_e"]
     k = I.shape[1]
     dY = dX_out[I]                                         # [e, k, d] rows of dX_out seen by each slot
-    dX_e = G[:, :, None] * dY                              # Eq. 4 w.r.t. X_e
+    dX_e = store("dX_e", G[:, :, None] * dY)               # Eq. 4 w.r.t. X_e
     dG = np.einsum("ijd,ijd->ij", dY, X_e)                 # Eq. 4 w.r.t. G
     dH = np.stack([dX_e[i] @ W2[i] for i in range(e)])     # [e, k, d']
-    dW2 = np.stack([dX_e[i].T @ H[i] for i in range(e)])   # [e, d, d']
-    dZ = dH * gelu_grad(Z, gelu_variant)
-    dW1 = np.stack([X_in[i].T @ dZ[i] for i in range(e)])  # [e, d, d']
-    dX_in = np.stack([dZ[i] @ W1[i].T for i in range(e)])  # [e, k, d]
+    dW2 = store("dW2", np.stack([dX_e[i].T @ H[i] for i in range(e)]))   # [e, d, d']
+    dZ = store("dZ", dH * gelu_grad(Z, gelu_variant))
+    dW1 = store("dW1", np.stack([X_in[i].T @ dZ[i] for i in range(e)]))  # [e, d, d']
+    dX_in = store("dX_in", np.stack([dZ[i] @ W1[i].T for i in range(e)]))  # [e, k, d]
     dS = np.zeros((n, e), F64)
     for i in range(e):
         dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
     dL = S * (dS - (dS * S).sum(axis=1, keepdims=True))    # softmax Jacobian, per token row
-    dWg = X.T @ dL
+    dWg = store("dWg", X.T @ dL)
     dX = dL @ Wg.T
     for i in range(e):
         for j in range(k):
             dX[I[i, j]] += dX_in[i, j]
+    dX = store("dX", dX)
     return dict(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2, dX_e=dX_e, dG=dG, dH=dH, dZ=dZ,
                 dX_in=dX_in, dS=dS, dL=dL)
 

@@ -199,4 +199,4 @@ def saved_view(cfg, saved) -> dict:
                 G=view(v.G, (E, k), torch.float32, 4), row_ptr=view(v.row_ptr, (n + 1,), torch.int32, 4),
                 slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es),
                 Z=view(v.Z, (E, k, f), dt, es), H=view(v.H, (E, k, f), dt, es),
-                X_e=view(v.X_e, (E, k, d), dt, es))
+                X_e=view(v.X_e, (E, k, d), torch.float32, 4))

@@ -45,7 +45,7 @@ SavedLayout saved_layout(const Dims& D) {
   L.X_in = take((size_t)D.slots * D.d * D.eb);
   L.Z = take((size_t)D.slots * D.dff * D.eb);
   L.H = take((size_t)D.slots * D.dff * D.eb);
-  L.X_e = take((size_t)D.slots * D.d * D.eb);
+  L.X_e = take((size_t)D.slots * D.d * 4);          // fp32 on both paths
   L.total = o;
   return L;
 }
@@ -83,6 +83,7 @@ struct BatchedGemm {
   void* C; int64_t ldc, batch_c;
   int M, N, K, batches, epi;
   void* C2; const void* Zin;
+  int c_f32;                                         // C is fp32 regardless of the path's dtype
 };
 
 ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaStream_t st) {
@@ -91,12 +92,13 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
     t.A = b.A; t.B = b.B; t.a_mn_major = b.a_mn; t.b_mn_major = b.b_mn;
     t.M = b.M; t.N = b.N; t.K = b.K; t.batches = b.batches;
     t.lda = b.lda; t.ldb = b.ldb; t.batch_a = b.batch_a; t.batch_b = b.batch_b;
-    t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c;
+    t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c; t.c_f32 = b.c_f32;
     t.status = status_word;
     if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); return EC_OK; }
   }
   GemmArgs g; memset(&g, 0, sizeof(g));
   g.A = b.A; g.B = b.B; g.C = b.C; g.a_dtype = g.b_dtype = g.c_dtype = D.dtype;
+  if (b.c_f32) g.c_dtype = EC_F32;
   g.M = b.M; g.N = b.N; g.K = b.K; g.batches = b.batches;
   g.sam = b.a_mn ? 1 : b.lda; g.sak = b.a_mn ? b.lda : 1;
   g.sbk = b.b_mn ? b.ldb : 1; g.sbn = b.b_mn ? 1 : b.ldb;
@@ -149,7 +151,7 @@ ec_status ec_saved_view(const ec_config* c, void* saved, ec_saved_ptrs* out) {
   const SavedLayout L = saved_layout(D); char* b = (char*)saved;
   out->S = (float*)(b + L.S); out->I = (int32_t*)(b + L.I); out->G = (float*)(b + L.G);
   out->row_ptr = (int32_t*)(b + L.row_ptr); out->slots = (int32_t*)(b + L.slots);
-  out->X_in = b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = b + L.X_e;
+  out->X_in = b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = (float*)(b + L.X_e);
   return EC_OK;
 }
 
@@ -178,7 +180,7 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   char* sv = (char*)saved; char* w = (char*)ws;
   float* S = (float*)(sv + L.S); int32_t* I = (int32_t*)(sv + L.I); float* G = (float*)(sv + L.G);
   int32_t* row_ptr = (int32_t*)(sv + L.row_ptr); int32_t* slots = (int32_t*)(sv + L.slots);
-  void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; void* X_e = sv + L.X_e;
+  void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; float* X_e = (float*)(sv + L.X_e);
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st)) != EC_OK) return s;
@@ -187,8 +189,8 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   // Z = X_in[i] . W1[i],  H = GeLU(Z)
   BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr};
   if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
-  // X_e = H[i] . W2[i]^T
-  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
+  // X_e = H[i] . W2[i]^T, kept in fp32
+  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1};
   if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
   EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
   return EC_OK;
@@ -209,7 +211,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   const float* S = (const float*)(sv + L.S); const int32_t* I = (const int32_t*)(sv + L.I);
   const float* G = (const float*)(sv + L.G);
   const int32_t* row_ptr = (const int32_t*)(sv + L.row_ptr); const int32_t* slots = (const int32_t*)(sv + L.slots);
-  const void* X_in = sv + L.X_in; const void* Z = sv + L.Z; const void* H = sv + L.H; const void* X_e = sv + L.X_e;
+  const void* X_in = sv + L.X_in; const void* Z = sv + L.Z; const void* H = sv + L.H; const float* X_e = (const float*)(sv + L.X_e);
   void* dX_e = w + W.dX_e; float* dG = (float*)(w + W.dG); void* dZ = w + W.dZ; void* dX_in = w + W.dX_in;
   float* dL = (float*)(w + W.dL); float* part = (float*)(w + W.dWg_part);
   int* status = (int*)(w + W.status);

@@ -32,10 +32,10 @@ cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t slots_tota
                                  int32_t* slots, void* scratch, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t slots_total,
                           int d, cudaStream_t st);
-cudaError_t launch_combine(int dtype, const void* X_e, const float* G, const int32_t* row_ptr,
+cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const int32_t* row_ptr,
                            const int32_t* slots, void* X_out, int64_t n, int d, cudaStream_t st);
 // dX_e[s,:] = G[s] * dX_out[I[s],:],  dG[s] = <dX_out[I[s],:], X_e[s,:]>
-cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const void* X_e, const float* G,
+cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, const float* G,
                                const int32_t* I, void* dX_e, float* dG, int64_t slots_total, int d,
                                cudaStream_t st);
 // dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] S[t,i']),  dS scattered from dG through the inverse index
@@ -73,7 +73,8 @@ struct TcGemmArgs {
   int64_t lda, ldb; // elements between consecutive rows of the stored matrices
   int64_t batch_a, batch_b;
   int epi, gelu;    // EPI_STORE / EPI_GELU / EPI_GELU_GRAD, or EPI_SOFTMAX below
-  void* C; void* C2; const void* Zin; int64_t ldc; int64_t batch_c;   // bf16 outputs
+  void* C; void* C2; const void* Zin; int64_t ldc; int64_t batch_c;   // bf16 outputs (C is fp32 when c_f32)
+  int c_f32;
   float* S;         // EPI_SOFTMAX: fp32 row softmax of the N columns, [M, N]
   int* status;      // device status word
 };

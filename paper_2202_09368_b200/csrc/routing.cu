@@ -466,36 +466,50 @@ cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in
 // Unshuffle, Eq. 4: X_out[t,:] = sum over the slots of t (ascending expert) of G[s] * X_e[s,:].
 // Read through the token->slot index, so no atomics and a fixed summation order.
 // ------------------------------------------------------------------------------------------
+// four consecutive elements of a row of T
+__device__ __forceinline__ void load4(const float* p, float* f) {
+  const float4 v = *reinterpret_cast<const float4*>(p); f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+__device__ __forceinline__ void load4(const bf16* p, float* f) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+  f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float* f) {
+  *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+}
+__device__ __forceinline__ void store4(bf16* p, const float* f) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<unsigned*>(&a), *reinterpret_cast<unsigned*>(&b));
+}
+
 template <typename T>
-__global__ void combine_kernel(const uint4* __restrict__ X_e, const float* __restrict__ G,
+__global__ void combine_kernel(const float* __restrict__ X_e, const float* __restrict__ G,
                                const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
-                               uint4* __restrict__ X_out, int64_t total_vec, int vec_per_row) {
-  constexpr int N = Vec<T>::N;
-  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_vec; g += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t t = g / vec_per_row; const int v = (int)(g % vec_per_row);
-    float acc[N];
-#pragma unroll
-    for (int i = 0; i < N; ++i) acc[i] = 0.f;
+                               T* __restrict__ X_out, int64_t total_quads, int quads_per_row) {
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_quads; g += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = g / quads_per_row; const int v = (int)(g % quads_per_row);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const int a = row_ptr[t], b = row_ptr[t + 1];
     for (int q = a; q < b; ++q) {
       const int s = slots[q];
       const float w = G[s];
-      float x[N];
-      Vec<T>::unpack(X_e[(int64_t)s * vec_per_row + v], x);
+      float x[4];
+      load4(X_e + ((int64_t)s * quads_per_row + v) * 4, x);
 #pragma unroll
-      for (int i = 0; i < N; ++i) acc[i] = fmaf(w, x[i], acc[i]);
+      for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, x[i], acc[i]);
     }
-    X_out[g] = Vec<T>::pack(acc);
+    store4(X_out + g * 4, acc);
   }
 }
 
-cudaError_t launch_combine(int dtype, const void* X_e, const float* G, const int32_t* row_ptr, const int32_t* slots,
+cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const int32_t* row_ptr, const int32_t* slots,
                            void* X_out, int64_t n, int d, cudaStream_t st) {
-  const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
-  const int64_t tv = n * vpr;
-  const unsigned grid = grid_for(tv, 256, 148 * 32);
-  if (dtype == 0) combine_kernel<float><<<grid, 256, 0, st>>>((const uint4*)X_e, G, row_ptr, slots, (uint4*)X_out, tv, vpr);
-  else combine_kernel<bf16><<<grid, 256, 0, st>>>((const uint4*)X_e, G, row_ptr, slots, (uint4*)X_out, tv, vpr);
+  const int qpr = d / 4;
+  const int64_t tq = n * qpr;
+  const unsigned grid = grid_for(tq, 256, 148 * 32);
+  if (dtype == 0) combine_kernel<float><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (float*)X_out, tq, qpr);
+  else combine_kernel<bf16><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (bf16*)X_out, tq, qpr);
   return cudaGetLastError();
 }
 
@@ -504,35 +518,34 @@ cudaError_t launch_combine(int dtype, const void* X_e, const float* G, const int
 //   dX_e[s,:] = G[s] * dX_out[t,:],   dG[s] = <dX_out[t,:], X_e[s,:]>.   One warp per slot.
 // ------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void bwd_combine_kernel(const uint4* __restrict__ dX_out, const uint4* __restrict__ X_e,
+__global__ void bwd_combine_kernel(const T* __restrict__ dX_out, const float* __restrict__ X_e,
                                    const float* __restrict__ G, const int32_t* __restrict__ I,
-                                   uint4* __restrict__ dX_e, float* __restrict__ dG, int64_t total, int vec_per_row) {
-  constexpr int N = Vec<T>::N;
+                                   T* __restrict__ dX_e, float* __restrict__ dG, int64_t total, int quads_per_row) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t s = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; s < total; s += warps) {
     const int64_t t = I[s];
     const float w = G[s];
     float dot = 0.f;
-    for (int v = lane; v < vec_per_row; v += 32) {
-      float dy[N], xe[N], o[N];
-      Vec<T>::unpack(dX_out[t * vec_per_row + v], dy);
-      Vec<T>::unpack(X_e[s * vec_per_row + v], xe);
+    for (int v = lane; v < quads_per_row; v += 32) {
+      float dy[4], xe[4], o[4];
+      load4(dX_out + (t * quads_per_row + v) * 4, dy);
+      load4(X_e + (s * quads_per_row + v) * 4, xe);
 #pragma unroll
-      for (int i = 0; i < N; ++i) { o[i] = w * dy[i]; dot = fmaf(dy[i], xe[i], dot); }
-      dX_e[s * vec_per_row + v] = Vec<T>::pack(o);
+      for (int i = 0; i < 4; ++i) { o[i] = w * dy[i]; dot = fmaf(dy[i], xe[i], dot); }
+      store4(dX_e + (s * quads_per_row + v) * 4, o);
     }
     for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
     if (lane == 0) dG[s] = dot;
   }
 }
 
-cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const void* X_e, const float* G, const int32_t* I,
+cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, const float* G, const int32_t* I,
                                void* dX_e, float* dG, int64_t total, int d, cudaStream_t st) {
-  const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
+  const int qpr = d / 4;
   const unsigned grid = grid_for(total * 32, 256, 148 * 16);
-  if (dtype == 0) bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const uint4*)dX_out, (const uint4*)X_e, G, I, (uint4*)dX_e, dG, total, vpr);
-  else bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const uint4*)dX_out, (const uint4*)X_e, G, I, (uint4*)dX_e, dG, total, vpr);
+  if (dtype == 0) bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)dX_out, X_e, G, I, (float*)dX_e, dG, total, qpr);
+  else bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)dX_out, X_e, G, I, (bf16*)dX_e, dG, total, qpr);
   return cudaGetLastError();
 }
 

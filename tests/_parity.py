@@ -7,7 +7,14 @@ compare it with the CPU oracle following the protocol
   (iii) every later tensor against the oracle evaluated with S and I fixed to the
         GPU's (a one-ulp difference in S may legitimately flip a boundary token).
 
-Error measure: max|gpu - ref| / RMS(ref), per tensor.
+Error measure: max|gpu - ref| / RMS(ref), per tensor.  Bound: 1e-4 on the fp32 path.
+On the bf16 path the bound is 2e-2, except where the storage format alone already
+costs more: the layer keeps Z, H, dX_e, dZ, dX_in and its outputs in bf16 (they
+are tensor-core operands or bf16 activations by definition of the path), and its
+outputs are heavy-tailed (a token's row scales with its gate weights), so the
+exact fp64 result rounded once to bf16 can sit above 2e-2 by itself.  The test
+therefore also evaluates the oracle with those tensors rounded to bf16 where they
+are stored (the arithmetic floor, CPU only) and accepts max(2e-2, 1.5 x floor).
 """
 import numpy as np
 import torch
@@ -24,6 +31,16 @@ def rel_err(got, ref):
     if rms == 0:
         return float(np.max(np.abs(got)))
     return float(np.max(np.abs(got - ref)) / rms)
+
+
+BF16_STORED = {"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dX", "dWg", "dW1", "dW2"}
+
+
+def bf16_store(name, x):
+    """Storage rounding of the bf16 path: round-to-nearest-even to bf16 where the layer keeps bf16."""
+    if name not in BF16_STORED:
+        return x
+    return torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
 
 
 def to_np(t):
@@ -74,6 +91,16 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         b = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), f, gelu)
         for name, t in (("dX", dX), ("dWg", dWg), ("dW1", dW1), ("dW2", dW2)):
             errs[name] = rel_err(to_np(t), b[name])
-    bad = {k_: e for k_, e in errs.items() if not e <= tol}
-    assert not bad, f"over tolerance {tol}: {bad} (all: {errs})"
+    bound = {k_: tol for k_ in errs}
+    if dtype == torch.bfloat16:
+        ff = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(),
+                       store=bf16_store)
+        floor = {k_: rel_err(ff[k_], f[k_]) for k_ in ("Z", "H", "X_e", "X_out")}
+        if backward:
+            fb = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), ff, gelu, store=bf16_store)
+            floor.update({k_: rel_err(fb[k_], b[k_]) for k_ in ("dX", "dWg", "dW1", "dW2")})
+        bound = {k_: max(tol, 1.5 * floor.get(k_, 0.0)) for k_ in errs}
+        errs["_floor"] = floor
+    bad = {k_: (e, bound[k_]) for k_, e in errs.items() if k_ in bound and not e <= bound[k_]}
+    assert not bad, f"over tolerance (err, bound): {bad} (all: {errs})"
     return errs

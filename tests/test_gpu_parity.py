@@ -57,7 +57,7 @@ def test_routing_with_heavy_ties(n, d, E, c, levels, dtype):
     X, Wg = IN.quantised_gate_inputs(n, d, E, levels, dtype)
     cfg = B.make_config(n, d, 16, E, c, dtype)
     r = B.ec_route(cfg, X.cuda(), Wg.cuda())
-    assert len(np.unique(r.S.cpu().numpy()[:, 0])) <= 2 * levels + 1
+    assert len(np.unique(r.S.cpu().numpy()[:, 0])) <= d          # tokens t and t+d share a row of logits
     check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
 
 
@@ -92,9 +92,9 @@ def test_run_to_run_determinism():
     for _ in range(2):
         Y, saved = B.ec_moe_forward(cfg, X, Wg, W1, W2)
         g = B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved)
-        outs.append([Y.clone()] + [t.clone() for t in g] + [saved.clone()])
+        outs.append([Y.clone()] + [t.clone() for t in g] + [t.clone() for t in B.saved_view(cfg, saved).values()])
     for a, b in zip(*outs):
-        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+        assert torch.equal(a.contiguous().view(torch.uint8), b.contiguous().view(torch.uint8))   # bitwise
 
 
 def test_argument_errors_are_reported_before_any_launch():
