@@ -1,0 +1,320 @@
+"""Benchmark of the expert-choice MoE layer (forward + backward) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4|cfg2|small] [--impl reference]
+
+A step is one forward + backward pass of the whole layer over one group of n tokens
+(routing, gather, expert FFNs, combine, and every backward kernel).  Prints ONE JSON
+line.  `value` is tokens/s with all inputs resident in HBM; `e2e` is the same metric
+with the step's inputs (X, dX_out) copied from pinned host memory and its results
+(X_out, dX) copied back inside the timed region.  With N > 1 (torchrun) every rank
+runs its own group on its own GPU: the layer routes each group independently, there
+is no data-path collective, and the ranks are replicas (weak scaling).
+
+`--impl reference` times the CPU oracle (fp64 numpy, as it stands) on the host cores
+on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (n, d, d', E, c)   shapes of Table 1 at sequence length 1024
+    "cfg4": (16384, 4096, 16384, 64, 2.0),      # 8B/64E-shaped layer (headline)
+    "cfg2": (8192, 768, 3072, 32, 2.0),         # 100M/32E-shaped layer
+    "small": (2048, 256, 512, 8, 2.0),
+}
+GEMM_STAGES = ("gemm1_gelu", "gemm2", "gemm_dZ", "gemm_dW2", "gemm_dW1", "gemm_dXin")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            j = json.load(f)
+        return dict(hbm_gbs=j["hbm_gbs"], tflops_burst=j["bf16_tflops"],
+                    tflops_sustained=j["bf16_tflops_sustained"], source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], 0, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = max(mx, float(r[1]))
+                for nme, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nme)
+            except Exception:
+                pass
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def layer_flops(n, d, dff, E, c):
+    slots = int(n * c)
+    gemm = 2.0 * slots * d * dff                 # one expert-batched GEMM
+    gate = 2.0 * n * d * E
+    return dict(gemm=gemm, fwd=2 * gemm + gate, bwd=4 * gemm + 2 * gate)
+
+
+# ----------------------------------------------------------------------------------- CPU oracle timing
+def time_oracle_sample(n, d, dff, E, c, seed=0, experts=1):
+    """Times the oracle on routing in full plus `experts` whole experts forward + backward and
+    extrapolates the expert part to E experts.  Returns (tokens/s, threads, description)."""
+    import numpy as np
+    import torch
+    from oracle import ec_oracle as O
+    from paper_2202_09368_b200 import inputs as IN
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    bf = torch.bfloat16
+    X = IN.normal_tensor((n, d), 1.0, seed, IN.TID_X, bf).float().numpy().astype(np.float64)
+    Wg = IN.normal_tensor((d, E), 1.0 / math.sqrt(d), seed, IN.TID_WG, bf).float().numpy().astype(np.float64)
+    dY = IN.normal_tensor((n, d), 1.0, seed, IN.TID_DXOUT, bf).float().numpy().astype(np.float64)
+    per = d * dff
+    W1 = [(IN.normal_chunk(seed, IN.TID_W1, i * per, per) / math.sqrt(d)).to(bf).float().numpy().astype(np.float64).reshape(d, dff)
+          for i in range(experts)]
+    W2 = [(IN.normal_chunk(seed, IN.TID_W2, i * per, per) / math.sqrt(dff)).to(bf).float().numpy().astype(np.float64).reshape(d, dff)
+          for i in range(experts)]
+    t0 = time.perf_counter()
+    r = O.route(X, Wg, c)
+    t_route = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for i in range(experts):
+        I_i, G_i = r["I"][i], r["G"][i]
+        X_in = X[I_i]
+        Z, H, X_e = O.expert_ffn(X_in, W1[i], W2[i])
+        dX_e = G_i[:, None] * dY[I_i]
+        dG = np.einsum("jd,jd->j", dY[I_i], X_e)
+        O.expert_ffn_backward(dX_e, X_in, Z, H, W1[i], W2[i])
+    t_exp = (time.perf_counter() - t0) / experts
+    total = t_route + E * t_exp
+    what = (f"oracle (numpy fp64) on n={n} d={d} d'={dff} E={E} c={c}: routing in full ({t_route:.2f} s) + "
+            f"{experts} of {E} experts forward+backward ({t_exp:.2f} s each), expert part extrapolated x{E}; "
+            f"combine and gate backward not included")
+    return n / total, threads, what
+
+
+def run_reference(args):
+    n, d, dff, E, c = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(max(1, min(args.steps, 2))):          # bounded: each step is seconds of CPU work
+        v, threads, what = time_oracle_sample(n, d, dff, E, c)
+        vals.append(v)
+    v = sum(vals) / len(vals)
+    out = {"impl": "reference", "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": v, "unit": "tokens/s",
+           "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / v,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{args.workload}: n={n} d={d} d_ff={dff} E={E} c={c}"},
+           "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
+           "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+# ----------------------------------------------------------------------------------- GPU arm
+def aggregate_max(t_local_ms: float, device) -> float:
+    """Max over ranks of a per-rank time (one all-reduce on the bench's process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return t_local_ms
+    t = torch.tensor([t_local_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2202_09368_b200 import binding as B
+    from paper_2202_09368_b200 import inputs as IN
+
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    n, d, dff, E, c = WORKLOADS[args.workload]
+    bf = torch.bfloat16
+    cfg = B.make_config(n, d, dff, E, c, bf)
+    seed = rank                                                   # each rank routes its own group
+    chunk = 1 << 26
+    X = IN.normal_tensor((n, d), 1.0, seed, IN.TID_X, bf, dev, chunk)
+    Wg = IN.normal_tensor((d, E), 1.0 / math.sqrt(d), seed, IN.TID_WG, bf, dev, chunk)
+    W1 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(d), seed, IN.TID_W1, bf, dev, chunk)
+    W2 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(dff), seed, IN.TID_W2, bf, dev, chunk)
+    dY = IN.normal_tensor((n, d), 1.0, seed, IN.TID_DXOUT, bf, dev, chunk)
+    ws = B.alloc_workspace(cfg, dev); saved = B.alloc_saved(cfg, dev)
+    X_out = torch.empty_like(X)
+    grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
+
+    def step():
+        B.ec_moe_forward(cfg, X, Wg, W1, W2, X_out, saved, ws)
+        B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, grads, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    assert B.ec_read_status(ws) == B.EC_OK
+    # ---- timed region: K steps, device timed, max over ranks
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = B.ec_launch_count()
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        barrier()
+    launches = B.ec_launch_count() - l0
+    ms_total = aggregate_max(ev0.elapsed_time(ev1), dev)
+    ms_step = ms_total / args.steps
+    assert B.ec_read_status(ws) == B.EC_OK
+
+    # ---- per-stage times (CUDA events recorded by the library on the launching stream)
+    B.ec_profile_enable(True)
+    stage_ms = {}
+    reps = min(args.steps, 5)
+    for _ in range(reps):
+        B.ec_moe_forward(cfg, X, Wg, W1, W2, X_out, saved, ws)
+        for k_, v_ in B.ec_profile_read():
+            stage_ms[k_] = stage_ms.get(k_, 0.0) + v_ / reps
+        B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, grads, ws)
+        for k_, v_ in B.ec_profile_read():
+            stage_ms[k_] = stage_ms.get(k_, 0.0) + v_ / reps
+    B.ec_profile_enable(False)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    hX, hdY = X.cpu().pin_memory(), dY.cpu().pin_memory()
+    hOut, hdX = torch.empty_like(hX).pin_memory(), torch.empty_like(hX).pin_memory()
+    dXin_dev, dYin_dev = torch.empty_like(X), torch.empty_like(dY)
+
+    def e2e_step():
+        dXin_dev.copy_(hX, non_blocking=True); dYin_dev.copy_(hdY, non_blocking=True)
+        B.ec_moe_forward(cfg, dXin_dev, Wg, W1, W2, X_out, saved, ws)
+        B.ec_moe_backward(cfg, dXin_dev, Wg, W1, W2, dYin_dev, saved, grads, ws)
+        hOut.copy_(X_out, non_blocking=True); hdX.copy_(grads[0], non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e_steps = max(1, min(args.steps, 10))
+    ev0.record()
+    for _ in range(e_steps):
+        e2e_step()
+    ev1.record()
+    barrier()
+    e2e_ms = aggregate_max(ev0.elapsed_time(ev1), dev) / e_steps
+    io_bytes = X.numel() * 2 * 2
+
+    fl = layer_flops(n, d, dff, E, c)
+    peaks = measured_peaks()
+    gemm_ms = [stage_ms[s] for s in GEMM_STAGES if s in stage_ms]
+    gemm_avg_ms = sum(gemm_ms) / max(1, len(gemm_ms))
+    achieved = fl["gemm"] / (gemm_avg_ms * 1e-3) / 1e12 if gemm_ms else None
+    peak = peaks["tflops_sustained"]
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            v, threads, what = time_oracle_sample(n, d, dff, E, c)
+            cpu = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what}
+        out = {
+            "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": world * n / (ms_step * 1e-3), "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} "
+                                   f"fwd+bwd, bf16 storage / fp32 accumulate, one routing group per GPU",
+                       "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
+                             if args.workload != "small" else "small case, L2 resident",
+                       "tensor_cores": bool(B.ec_uses_tensor_cores(cfg))},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": io_bytes,
+                    "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms},
+            "gpu_launches": launches,
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (6 launches per step: the expert GEMMs of Eq. 3 "
+                                                      "and their backward)",
+                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": (achieved / peak) if achieved else None,
+                         "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": None,
+                         "flops_per_launch": fl["gemm"], "avg_launch_ms": gemm_avg_ms},
+            "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
+            "layer_tflops": (fl["fwd"] + fl["bwd"]) / (ms_step * 1e-3) / 1e12,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -138,6 +138,22 @@ const char* ec_status_string(ec_status s);
  * kernels, 0 if it falls back to the plain FMA kernels (fp32 path, odd shapes). */
 int ec_uses_tensor_cores(const ec_config* cfg);
 
+/* Number of CUDA kernels this library has launched in this process so far (all calls, all
+ * streams).  The paper has no counterpart; benchmarks use the difference across a timed region. */
+long long ec_launch_count(void);
+
+/*
+ * Per-stage device timing, for benchmarks (no counterpart in the paper).  After
+ * ec_profile_enable(1), each call of ec_route / ec_moe_forward / ec_moe_backward records a CUDA
+ * event on its stream after every stage (gate, top-k, inverse index, gather, the GEMMs, combine,
+ * ...).  ec_profile_read waits for the last call's final event and writes up to max_stages
+ * elapsed times (milliseconds) and static stage names in launch order; it returns the number of
+ * stages, 0 when profiling is off, -1 on a CUDA error.  The state is global to the process: use
+ * it from one thread, one call at a time.  Off by default.
+ */
+void ec_profile_enable(int on);
+int ec_profile_read(float* ms, const char** names, int max_stages);
+
 #ifdef __cplusplus
 }
 #endif

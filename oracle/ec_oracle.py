@@ -32,6 +32,10 @@ from scipy.special import erf as _erf
 F64 = np.float64
 
 
+def _keep(name, x):
+    return x
+
+
 def capacity(n: int, c: float, e: int) -> int:
     """Eq. 1: k = n*c/e.  Non-integer values are floored; k < 1 or k > n is an error."""
     k = int(math.floor(n * float(c) / e + 1e-9))
@@ -105,6 +109,25 @@ def gelu_grad(z, variant: str = "erf"):
     raise ValueError(variant)
 
 
+def expert_ffn(X_in_i, W1_i, W2_i, gelu_variant: str = "erf", store=_keep):
+    """Eq. 3 for one expert: Z = X_in[i] . W1[i], H = GeLU(Z), X_e[i] = H . W2[i]^T."""
+    Z = X_in_i @ W1_i                                      # [k, d']
+    H = store("H", gelu(Z, gelu_variant))
+    Z = store("Z", Z)
+    X_e = store("X_e", H @ W2_i.T)                         # [k, d]
+    return Z, H, X_e
+
+
+def expert_ffn_backward(dX_e_i, X_in_i, Z_i, H_i, W1_i, W2_i, gelu_variant: str = "erf", store=_keep):
+    """Chain rule through Eq. 3 for one expert; returns dW1[i], dW2[i], dX_in[i], dH, dZ."""
+    dH = dX_e_i @ W2_i                                     # [k, d']
+    dW2 = store("dW2", dX_e_i.T @ H_i)                     # [d, d']
+    dZ = store("dZ", dH * gelu_grad(Z_i, gelu_variant))
+    dW1 = store("dW1", X_in_i.T @ dZ)                      # [d, d']
+    dX_in = store("dX_in", dZ @ W1_i.T)                    # [k, d]
+    return dW1, dW2, dX_in, dH, dZ
+
+
 def route(X, Wg, c: float, S_override=None):
     """Eq. 1-2: S, G, I and the token->slot inverse index."""
     n = np.asarray(X).shape[0]
@@ -114,10 +137,6 @@ def route(X, Wg, c: float, S_override=None):
     G, I = topk(S, k)
     row_ptr, slots = inverse_index(I, n)
     return dict(k=k, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots)
-
-
-def _keep(name, x):
-    return x
 
 
 def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
@@ -146,10 +165,10 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
         r.update(I=I, G=G, row_ptr=row_ptr, slots=slots)
     I, G = r["I"], r["G"]
     X_in = X[I]                                            # Eq. 3: X_in = P . X,  [e, k, d]
-    Z = np.stack([X_in[i] @ W1[i] for i in range(e)])      # [e, k, d']
-    H = store("H", gelu(Z, gelu_variant))
-    Z = store("Z", Z)
-    X_e = store("X_e", np.stack([H[i] @ W2[i].T for i in range(e)]))   # [e, k, d]
+    per_expert = [expert_ffn(X_in[i], W1[i], W2[i], gelu_variant, store) for i in range(e)]
+    Z = np.stack([p[0] for p in per_expert])               # [e, k, d']
+    H = np.stack([p[1] for p in per_expert])               # [e, k, d']
+    X_e = np.stack([p[2] for p in per_expert])             # [e, k, d]
     X_out = np.zeros((n, d), F64)                          # Eq. 4, experts in ascending order
     for i in range(e):
         for j in range(k):
@@ -173,11 +192,13 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     dY = dX_out[I]                                         # [e, k, d] rows of dX_out seen by each slot
     dX_e = store("dX_e", G[:, :, None] * dY)               # Eq. 4 w.r.t. X_e
     dG = np.einsum("ijd,ijd->ij", dY, X_e)                 # Eq. 4 w.r.t. G
-    dH = np.stack([dX_e[i] @ W2[i] for i in range(e)])     # [e, k, d']
-    dW2 = store("dW2", np.stack([dX_e[i].T @ H[i] for i in range(e)]))   # [e, d, d']
-    dZ = store("dZ", dH * gelu_grad(Z, gelu_variant))
-    dW1 = store("dW1", np.stack([X_in[i].T @ dZ[i] for i in range(e)]))  # [e, d, d']
-    dX_in = store("dX_in", np.stack([dZ[i] @ W1[i].T for i in range(e)]))  # [e, k, d]
+    per_expert = [expert_ffn_backward(dX_e[i], X_in[i], Z[i], H[i], W1[i], W2[i], gelu_variant, store)
+                  for i in range(e)]
+    dW1 = np.stack([p[0] for p in per_expert])             # [e, d, d']
+    dW2 = np.stack([p[1] for p in per_expert])             # [e, d, d']
+    dX_in = np.stack([p[2] for p in per_expert])           # [e, k, d]
+    dH = np.stack([p[3] for p in per_expert])
+    dZ = np.stack([p[4] for p in per_expert])
     dS = np.zeros((n, e), F64)
     for i in range(e):
         dS[I[i], i] = dG[i]                                # tokens of one expert are distinct

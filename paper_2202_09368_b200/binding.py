@@ -21,7 +21,7 @@ EC_GELU_ERF, EC_GELU_TANH = 0, 1
 
 EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
-           "ec_uses_tensor_cores"]
+           "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read"]
 
 
 class ec_config(C.Structure):
@@ -62,6 +62,10 @@ def lib():
         L.ec_read_status.restype = C.c_int; L.ec_read_status.argtypes = [V, V]
         L.ec_status_string.restype = C.c_char_p; L.ec_status_string.argtypes = [C.c_int]
         L.ec_uses_tensor_cores.restype = C.c_int; L.ec_uses_tensor_cores.argtypes = [P]
+        L.ec_launch_count.restype = C.c_longlong; L.ec_launch_count.argtypes = []
+        L.ec_profile_enable.restype = None; L.ec_profile_enable.argtypes = [C.c_int]
+        L.ec_profile_read.restype = C.c_int
+        L.ec_profile_read.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_char_p), C.c_int]
         _lib = L
     return _lib
 
@@ -176,6 +180,24 @@ def ec_moe_backward(cfg, X, Wg, W1, W2, dX_out, saved, grads=None, ws=None):
 
 def ec_read_status(ws) -> int:
     return int(lib().ec_read_status(_ptr(ws), _stream()))
+
+
+def ec_launch_count() -> int:
+    return int(lib().ec_launch_count())
+
+
+def ec_profile_enable(on: bool) -> None:
+    lib().ec_profile_enable(1 if on else 0)
+
+
+def ec_profile_read(max_stages: int = 20):
+    """[(stage name, milliseconds), ...] of the last profiled call."""
+    ms = (C.c_float * max_stages)()
+    names = (C.c_char_p * max_stages)()
+    cnt = lib().ec_profile_read(ms, names, max_stages)
+    if cnt < 0:
+        raise EcError(EC_ERR_CUDA, "ec_profile_read")
+    return [(names[i].decode(), float(ms[i])) for i in range(cnt)]
 
 
 def saved_view(cfg, saved) -> dict:

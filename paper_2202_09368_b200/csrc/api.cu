@@ -5,6 +5,7 @@
 
 #include <math.h>
 #include <string.h>
+#include <atomic>
 
 using namespace ecmoe;
 
@@ -76,6 +77,31 @@ inline bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)
 
 #define EC_CUDA(x) do { if ((x) != cudaSuccess) return EC_ERR_CUDA; } while (0)
 
+// Optional per-stage timing (ec_profile_enable): an event is recorded on the call's stream after
+// each stage of forward / backward.  Host state only; off by default and then free of cost.
+constexpr int kMaxStages = 20;
+struct Profile {
+  bool enabled = false;
+  cudaEvent_t ev[kMaxStages + 1];
+  bool created = false;
+  int count = 0;                       // stages recorded by the last call
+  const char* names[kMaxStages];
+};
+Profile g_prof;
+std::atomic<long long> g_launches{0};
+
+void prof_begin(cudaStream_t st) {
+  if (!g_prof.enabled) return;
+  if (!g_prof.created) { for (auto& e : g_prof.ev) cudaEventCreate(&e); g_prof.created = true; }
+  g_prof.count = 0;
+  cudaEventRecord(g_prof.ev[0], st);
+}
+void prof_mark(const char* name, cudaStream_t st) {
+  if (!g_prof.enabled || g_prof.count >= kMaxStages) return;
+  g_prof.names[g_prof.count] = name;
+  cudaEventRecord(g_prof.ev[++g_prof.count], st);
+}
+
 // One expert-batched GEMM: tensor cores when the shape allows, FMA otherwise.
 struct BatchedGemm {
   const void* A; int a_mn; int64_t lda, batch_a;     // a_mn = 0: A stored [M][K]; 1: stored [K][M]
@@ -119,12 +145,17 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
     if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); done = true; }
   }
   if (!done) EC_CUDA(launch_gate_softmax_simt(D.dtype, X, Wg, S, D.n, D.d, D.E, st));
+  prof_mark("gate_softmax", st);
   EC_CUDA(launch_topk(S, D.n, D.E, D.k, I, G, ws + W.topk, st));
+  prof_mark("topk", st);
   EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
+  prof_mark("inverse_index", st);
   return EC_OK;
 }
 
 }  // namespace
+
+namespace ecmoe { void count_launch(int n) { g_launches += n; } }
 
 extern "C" {
 
@@ -165,6 +196,7 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  prof_begin(st);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
 }
 
@@ -183,16 +215,21 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; float* X_e = (float*)(sv + L.X_e);
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  prof_begin(st);
   if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st)) != EC_OK) return s;
   EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
+  prof_mark("gather", st);
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Z = X_in[i] . W1[i],  H = GeLU(Z)
   BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr};
   if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
+  prof_mark("gemm1_gelu", st);
   // X_e = H[i] . W2[i]^T, kept in fp32
   BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1};
   if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
+  prof_mark("gemm2", st);
   EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
+  prof_mark("combine", st);
   return EC_OK;
 }
 
@@ -218,21 +255,28 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Eq. 4 backward: dX_e, dG
+  prof_begin(st);
   EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
+  prof_mark("bwd_combine", st);
   // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
   BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z};
   if ((s = run_gemm(D, g3, status, st)) != EC_OK) return s;
+  prof_mark("gemm_dZ", st);
   // dW2[i] = dX_e[i]^T . H[i]
   BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
   if ((s = run_gemm(D, g4, status, st)) != EC_OK) return s;
+  prof_mark("gemm_dW2", st);
   // dW1[i] = X_in[i]^T . dZ[i]
   BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
   if ((s = run_gemm(D, g5, status, st)) != EC_OK) return s;
+  prof_mark("gemm_dW1", st);
   // dX_in[i] = dZ[i] . W1[i]^T
   BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
   if ((s = run_gemm(D, g6, status, st)) != EC_OK) return s;
+  prof_mark("gemm_dXin", st);
   // softmax backward: dL [n, E] fp32
   EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, D.n, D.E, D.k, st));
+  prof_mark("bwd_softmax", st);
   // dWg = X^T . dL, split over the tokens into fixed chunks and summed in a fixed order
   {
     const int P = dwg_splits(D);
@@ -245,6 +289,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
     g.epi = EPI_STORE;
     EC_CUDA(launch_gemm_simt(g, st));
     EC_CUDA(launch_reduce_partials(D.dtype, part, dWg, P, (int64_t)D.d * D.E, st));
+    prof_mark("dWg", st);
   }
   // dX = dL . Wg^T + sum over the slots of each token of dX_in
   {
@@ -254,6 +299,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
     g.sam = D.E; g.sak = 1; g.sbk = 1; g.sbn = D.E; g.ldc = D.d;
     g.epi = EPI_ADD_SLOTS; g.row_ptr = row_ptr; g.slots = slots; g.rows = dX_in; g.ld_rows = D.d;
     EC_CUDA(launch_gemm_simt(g, st));
+    prof_mark("dX", st);
   }
   return EC_OK;
 }
@@ -276,6 +322,23 @@ const char* ec_status_string(ec_status s) {
     case EC_ERR_TIMEOUT: return "a bounded device-side wait expired";
   }
   return "unknown status";
+}
+
+long long ec_launch_count(void) { return g_launches.load(); }
+
+void ec_profile_enable(int on) { g_prof.enabled = on != 0; if (!on) g_prof.count = 0; }
+
+int ec_profile_read(float* ms, const char** names, int max_stages) {
+  if (!g_prof.enabled || g_prof.count == 0) return 0;
+  if (cudaEventSynchronize(g_prof.ev[g_prof.count]) != cudaSuccess) return -1;
+  int nst = g_prof.count < max_stages ? g_prof.count : max_stages;
+  for (int i = 0; i < nst; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_prof.ev[i], g_prof.ev[i + 1]) != cudaSuccess) return -1;
+    if (ms) ms[i] = t;
+    if (names) names[i] = g_prof.names[i];
+  }
+  return nst;
 }
 
 int ec_uses_tensor_cores(const ec_config* c) {

@@ -101,8 +101,8 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
 
 template <typename TA, typename TB>
 static void dispatch_c(const GemmArgs& g, dim3 grid, cudaStream_t st) {
-  if (g.c_dtype == 0) gemm_simt_kernel<TA, TB, float><<<grid, NT, 0, st>>>(g);
-  else gemm_simt_kernel<TA, TB, bf16><<<grid, NT, 0, st>>>(g);
+  if (g.c_dtype == 0) { count_launch(); gemm_simt_kernel<TA, TB, float><<<grid, NT, 0, st>>>(g); }
+  else { count_launch(); gemm_simt_kernel<TA, TB, bf16><<<grid, NT, 0, st>>>(g); }
 }
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {

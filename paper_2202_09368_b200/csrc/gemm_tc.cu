@@ -1,5 +1,444 @@
+// Batched bf16 GEMM on the 5th-generation tensor cores (tcgen05) for the expert FFNs (Eq. 3),
+// their backward contractions, and the gate of Eq. 2 (with the row softmax in the epilogue).
+//
+//   C[b] (M x N, fp32 accumulate) = A[b] (M x K) . B[b] (K x N),  b = 0 .. batches-1
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warp 0      TMA producer: fills a ring of shared-memory stages (A 128 x 64, B BN x 64 bf16,
+//               128-byte swizzle) with cp.async.bulk.tensor, one mbarrier per stage;
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M = 128, N = BN, K = 16) on shared-memory
+//               descriptors, accumulating in tensor memory; tcgen05.commit releases stages and
+//               publishes finished accumulators.  Two accumulators (2 x BN columns) are kept so the
+//               epilogue of one tile overlaps the main loop of the next;
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (one row of the tile per thread), apply the
+//               fused function (GeLU, GeLU', softmax), store.
+// Operands may be K-major (K contiguous in memory) or MN-major (M or N contiguous); the weights
+// W1, W2 [E, d, d'] and the activations are never transposed in memory, the shared-memory
+// descriptors carry the orientation.  Three-dimensional tensor maps (inner, rows, batch) let the
+// TMA unit zero-fill whatever a tile overhangs, so ragged M, N and K need no special code.
+// Tiles are ordered with M fastest so that CTAs running together share the same weight tile in L2.
+//
+// Every wait on an mbarrier is bounded: after about two seconds the kernel records
+// EC_ERR_TIMEOUT in the status word, all roles leave their loops and the CTA exits in order.
 #include "internal.h"
+
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <mutex>
+
 namespace ecmoe {
-bool tc_gemm_supported(const TcGemmArgs&) { return false; }
-cudaError_t launch_gemm_tc(const TcGemmArgs&, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int BM = 128, BK = 64, UK = 16;
+constexpr int kThreads = 192;
+constexpr int kABytes = BM * BK * 2;                 // 16 KiB
+constexpr int kSmemBudget = 200 * 1024;
+constexpr unsigned long long kWaitNs = 2000000000ull;
+
+__host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + bn * BK * 2; }
+__host__ __device__ constexpr int num_stages(int bn) { return kSmemBudget / stage_bytes(bn) > 8 ? 8 : kSmemBudget / stage_bytes(bn); }
+__host__ __device__ constexpr int tmem_cols(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }   // power of two for bn = 64, 128, 256
+
+struct TcParams {
+  int M, N, K, batches;
+  int a_mn, b_mn;
+  int tiles_m, tiles_n, total_tiles, kblocks;
+  int gelu;
+  bf16* C; bf16* C2; const bf16* Zin; float* Cf; float* S;
+  int64_t ldc, batch_c;
+  int* status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t spin = 1;; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if ((spin & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > kWaitNs) {
+        *abort_flag = 1;
+        atomicExch(status + 1, where);
+        atomicExch(status, 5 /* EC_ERR_TIMEOUT */);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float gelu_fwd(float z, int variant) {
+  if (variant == 0) return 0.5f * z * (1.f + erff(z * 0.70710678118654752f));
+  return 0.5f * z * (1.f + tanhf(0.7978845608028654f * (z + 0.044715f * z * z * z)));
+}
+__device__ __forceinline__ float gelu_bwd(float z, int variant) {
+  if (variant == 0)
+    return 0.5f * (1.f + erff(z * 0.70710678118654752f)) + z * 0.3989422804014327f * __expf(-0.5f * z * z);
+  const float a = 0.7978845608028654f;
+  const float th = tanhf(a * (z + 0.044715f * z * z * z));
+  return 0.5f * (1.f + th) + 0.5f * z * (1.f - th * th) * a * (1.f + 3.f * 0.044715f * z * z);
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  __nv_bfloat162 p0 = __floats2bfloat162_rn(f[0], f[1]), p1 = __floats2bfloat162_rn(f[2], f[3]);
+  __nv_bfloat162 p2 = __floats2bfloat162_rn(f[4], f[5]), p3 = __floats2bfloat162_rn(f[6], f[7]);
+  return make_uint4(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1),
+                    *reinterpret_cast<unsigned*>(&p2), *reinterpret_cast<unsigned*>(&p3));
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  constexpr int S = num_stages(BN);
+  constexpr int kBBytes = BN * BK * 2;
+  constexpr int kStage = kABytes + kBBytes;
+  constexpr int kCols = tmem_cols(BN);
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = (uint64_t*)(smem + S * kStage);          // full[S], empty[S], tmem_full[2], tmem_empty[2]
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * S + 4);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+  const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, tfull0 = empty0 + 8 * S, tempty0 = tfull0 + 16;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 128); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t smem_base = smem_u32(smem);
+  bool gave_up = false;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && !gave_up; tile += gridDim.x) {
+        const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
+        const int m0 = mt * BM, n0 = nt * BN;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
+          const uint32_t bar = full0 + 8 * stage;
+          const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
+          mbar_expect_tx(bar, kStage);
+          const int k0 = kb * BK;
+          if (p.a_mn) {                       // stored [K][M]: boxes of 64 (M) x 64 (K)
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
+          } else {                            // stored [M][K]: one box 64 (K) x 128 (M)
+            tma_load_3d(sa, &tmA, bar, k0, m0, b);
+          }
+          if (p.b_mn) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+          } else {
+            tma_load_3d(sb, &tmB, bar, k0, n0, b);
+          }
+          if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // K-major: 8-row groups 1024 B apart, 32 B per K step inside the swizzle atom.
+      // MN-major: 64-wide blocks BK*128 B apart (LBO), 8-row K groups 1024 B apart (SBO), 2 groups per K step.
+      const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
+      const uint32_t a_step = p.a_mn ? 2048 : 32, b_step = p.b_mn ? 2048 : 32;
+      int stage = 0; uint32_t phase = 0; int it = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && !gave_up; tile += gridDim.x, ++it) {
+        const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
+        if (!mbar_wait(tempty0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.status, 2)) { gave_up = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3)) { gave_up = true; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
+#pragma unroll
+          for (int kk = 0; kk < BK / UK; ++kk) {
+            const uint64_t ad = make_desc(sa + kk * a_step, a_lbo, 1024);
+            const uint64_t bd = make_desc(sb + kk * b_step, b_lbo, 1024);
+            tc_mma(d_tmem, ad, bd, idesc, (kb | kk) != 0);
+          }
+          tc_commit(empty0 + 8 * stage);           // stage is free once these MMAs have read it
+          if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+        if (!gave_up) tc_commit(tfull0 + 8 * buf); // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue, one tile row per thread
+    const int q = warp & 3;                        // TMEM lane quarter this warp may read
+    int it = 0;
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++it) {
+      const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
+      const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
+      const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
+      if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
+      tc_fence_after();
+      const int row = mt * BM + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
+      const int n0 = nt * BN;
+      const int64_t obase = (int64_t)b * p.batch_c + (int64_t)row * p.ldc;
+      if constexpr (EPI == EPI_SOFTMAX) {
+        // Eq. 2: softmax over the N = E columns of this row; columns >= N are padding.
+        float mx = -INFINITY;
+        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
+          uint32_t r[32]; tc_ld32(taddr + c0, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (c0 + j < p.N) mx = fmaxf(mx, __uint_as_float(r[j]));
+        }
+        float sum = 0.f;
+        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
+          uint32_t r[32]; tc_ld32(taddr + c0, r);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (c0 + j < p.N) sum += expf(__uint_as_float(r[j]) - mx);
+        }
+        const float inv = 1.f / sum;
+        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
+          uint32_t r[32]; tc_ld32(taddr + c0, r);
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              if (c0 + j < p.N) {          // N is a multiple of 8
+                float4 o;
+                o.x = expf(__uint_as_float(r[j]) - mx) * inv; o.y = expf(__uint_as_float(r[j + 1]) - mx) * inv;
+                o.z = expf(__uint_as_float(r[j + 2]) - mx) * inv; o.w = expf(__uint_as_float(r[j + 3]) - mx) * inv;
+                *reinterpret_cast<float4*>(p.S + (int64_t)row * p.ldc + c0 + j) = o;
+              }
+            }
+          }
+        }
+      } else {
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          if (n0 + c0 >= p.N) break;               // uniform across the warp
+          uint32_t r[32]; tc_ld32(taddr + c0, r);
+          if (!row_ok) continue;
+          const int64_t o = obase + n0 + c0;
+          if constexpr (EPI == EPI_STORE) {
+            if (p.Cf) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                if (n0 + c0 + j < p.N)
+                  *reinterpret_cast<float4*>(p.Cf + o + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                         __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                if (n0 + c0 + j < p.N) {
+                  float f[8];
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[j + e]);
+                  *reinterpret_cast<uint4*>(p.C + o + j) = pack8(f);
+                }
+              }
+            }
+          } else if constexpr (EPI == EPI_GELU) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              if (n0 + c0 + j < p.N) {
+                float z[8], h[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[j + e]); h[e] = gelu_fwd(z[e], p.gelu); }
+                *reinterpret_cast<uint4*>(p.C + o + j) = pack8(z);
+                *reinterpret_cast<uint4*>(p.C2 + o + j) = pack8(h);
+              }
+            }
+          } else if constexpr (EPI == EPI_GELU_GRAD) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              if (n0 + c0 + j < p.N) {
+                const uint4 zv = *reinterpret_cast<const uint4*>(p.Zin + o + j);
+                const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w};
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float z0 = __uint_as_float(zw[e] << 16), z1 = __uint_as_float(zw[e] & 0xFFFF0000u);
+                  f[2 * e] = __uint_as_float(r[j + 2 * e]) * gelu_bwd(z0, p.gelu);
+                  f[2 * e + 1] = __uint_as_float(r[j + 2 * e + 1]) * gelu_bwd(z1, p.gelu);
+                }
+                *reinterpret_cast<uint4*>(p.C + o + j) = pack8(f);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty0 + 8 * buf);              // 128 arrivals free the accumulator
+    }
+  }
+
+  // ------------------------------------------------------------------ orderly exit
+  if (*abort_flag) {                               // let copies and MMAs still in flight drain
+    const unsigned long long t0 = globaltimer();
+    while (globaltimer() - t0 < 200000ull) __nanosleep(1000);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr; cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = (PFN_cuTensorMapEncodeTiled_v12000)p;
+  });
+  return fn;
+}
+
+// Tensor map over a bf16 matrix stored [batches][rows][inner] with row pitch ld and batch pitch bs (elements).
+bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, int64_t batches, int64_t ld, int64_t bs,
+              int box_inner, int box_rows) {
+  auto enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batches};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(batches > 1 ? bs : rows * ld) * 2};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_bn(const TcGemmArgs& g) { return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64); }
+
+template <int BN, int EPI>
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t st) {
+  constexpr int smem = num_stages(BN) * stage_bytes(BN) + 1024 + 256;
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  count_launch();
+  gemm_tc_kernel<BN, EPI><<<grid, kThreads, smem, st>>>(ta, tb, p);
+  return cudaGetLastError();
+}
+
+template <int EPI>
+cudaError_t launch_bn(int bn, const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t st) {
+  if (bn == 256) return launch_one<256, EPI>(ta, tb, p, st);
+  if (bn == 128) return launch_one<128, EPI>(ta, tb, p, st);
+  return launch_one<64, EPI>(ta, tb, p, st);
+}
+
+}  // namespace
+
+bool tc_gemm_supported(const TcGemmArgs& g) {
+  if (g.M < 1 || g.N < 1 || g.K < 1 || g.batches < 1) return false;
+  if (g.lda % 8 || g.ldb % 8 || g.ldc % 8 || g.N % 8) return false;            // 16-byte rows and vector stores
+  if (g.batches > 1 && (g.batch_a % 8 || g.batch_b % 8 || g.batch_c % 8)) return false;
+  if (((uintptr_t)g.A | (uintptr_t)g.B) & 15) return false;
+  if (g.epi == EPI_SOFTMAX && (g.N > 256 || g.batches != 1)) return false;
+  if ((int64_t)g.lda * 2 >= ((int64_t)1 << 40) || (int64_t)g.ldb * 2 >= ((int64_t)1 << 40)) return false;
+  return true;
+}
+
+cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
+  const int bn = pick_bn(g);
+  CUtensorMap ta, tb;
+  // A: K-major [M rows][K inner], box 64 x 128;  MN-major [K rows][M inner], box 64 x 64
+  const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, g.K, g.batches, g.lda, g.batch_a, 64, BK)
+                                : make_map(&ta, g.A, g.K, g.M, g.batches, g.lda, g.batch_a, BK, BM);
+  const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, g.K, g.batches, g.ldb, g.batch_b, 64, BK)
+                                : make_map(&tb, g.B, g.K, g.N, g.batches, g.ldb, g.batch_b, BK, bn);
+  if (!oka || !okb) return cudaErrorInvalidValue;
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.batches = g.batches; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
+  p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + bn - 1) / bn;
+  p.total_tiles = p.tiles_m * p.tiles_n * g.batches; p.kblocks = (g.K + BK - 1) / BK;
+  p.gelu = g.gelu;
+  p.C = g.c_f32 ? nullptr : (bf16*)g.C; p.Cf = g.c_f32 ? (float*)g.C : nullptr;
+  p.C2 = (bf16*)g.C2; p.Zin = (const bf16*)g.Zin; p.S = g.S;
+  p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
+  switch (g.epi) {
+    case EPI_STORE: return launch_bn<EPI_STORE>(bn, ta, tb, p, st);
+    case EPI_GELU: return launch_bn<EPI_GELU>(bn, ta, tb, p, st);
+    case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ta, tb, p, st);
+    case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ta, tb, p, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace ecmoe

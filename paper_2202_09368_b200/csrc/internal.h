@@ -20,6 +20,10 @@ struct StatusWord { int code; int where; int pad[62]; };
 // Per-expert state of the radix selection.
 struct SelState { unsigned long long prefix; unsigned int k_rem; unsigned int done; };
 
+// ---- bookkeeping (api.cu) ----------------------------------------------------------------------
+// Every kernel launch of the library goes through count_launch(); ec_launch_count() reports the sum.
+void count_launch(int n = 1);
+
 // ---- routing (routing.cu) -------------------------------------------------------------------
 cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, float* S, int64_t n,
                                      int d, int E, cudaStream_t st);

@@ -114,6 +114,7 @@ gate_softmax_simt_kernel(const T* __restrict__ X, const T* __restrict__ Wg, floa
 cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, float* S, int64_t n,
                                      int d, int E, cudaStream_t st) {
   const unsigned grid = (unsigned)((n + kGateTT - 1) / kGateTT);
+  count_launch();
   if (dtype == 0)
     gate_softmax_simt_kernel<float><<<grid, kGateThreads, 0, st>>>((const float*)X, (const float*)Wg, S, n, d, E);
   else
@@ -358,19 +359,27 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I,
   int64_t want = (int64_t)148 * 8 / L.chunks; if (want < 1) want = 1;
   int64_t rows = (n + want - 1) / want; if (rows < 64) rows = 64;
   const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks);
-  for (int pass = 0; pass < kRadixPasses; ++pass)
+  for (int pass = 0; pass < kRadixPasses; ++pass) {
+    count_launch();
     topk_hist_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
+  }
+  count_launch();
   topk_compact_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys);
   const int64_t tiles = (L.kpad + kSortTile - 1) / kSortTile;
   const unsigned sort_grid = (unsigned)(E * tiles);
   if (L.kpad <= kSortTile) {
+    count_launch();
     topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, L.kpad, 1, I, G);
   } else {
+    count_launch();
     topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, kSortTile, 0, I, G);
     const int64_t pairs = (int64_t)E * (L.kpad >> 1);
     for (int64_t size = 2 * kSortTile; size <= L.kpad; size <<= 1) {
-      for (int64_t stride = size >> 1; stride >= kSortTile; stride >>= 1)
+      for (int64_t stride = size >> 1; stride >= kSortTile; stride >>= 1) {
+        count_launch();
         topk_sort_global_kernel<<<grid_for(pairs, 256), 256, 0, st>>>(keys, L.kpad, pairs, size, stride);
+      }
+      count_launch();
       topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, size, size, size == L.kpad, I, G);
     }
   }
@@ -436,10 +445,14 @@ cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int
   cudaError_t e;
   // counts are built in slots' neighbour: reuse row_ptr[1..n] would break the scan, so count in `cursor`
   if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  count_launch();
   inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cursor);
+  count_launch();
   inv_scan_kernel<<<1, 1024, 0, st>>>(cursor, n, row_ptr);
   if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  count_launch();
   inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cursor, slots);
+  count_launch();
   inv_sort_kernel<<<grid_for(n, 256), 256, 0, st>>>(row_ptr, n, slots);
   return cudaGetLastError();
 }
@@ -458,6 +471,7 @@ __global__ void gather_kernel(const uint4* __restrict__ X, const int32_t* __rest
 cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t total, int d, cudaStream_t st) {
   const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
   const int64_t tv = total * vpr;
+  count_launch();
   gather_kernel<<<grid_for(tv, 256, 148 * 32), 256, 0, st>>>((const uint4*)X, I, (uint4*)X_in, tv, vpr);
   return cudaGetLastError();
 }
@@ -508,8 +522,8 @@ cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const in
   const int qpr = d / 4;
   const int64_t tq = n * qpr;
   const unsigned grid = grid_for(tq, 256, 148 * 32);
-  if (dtype == 0) combine_kernel<float><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (float*)X_out, tq, qpr);
-  else combine_kernel<bf16><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (bf16*)X_out, tq, qpr);
+  if (dtype == 0) { count_launch(); combine_kernel<float><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (float*)X_out, tq, qpr); }
+  else { count_launch(); combine_kernel<bf16><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (bf16*)X_out, tq, qpr); }
   return cudaGetLastError();
 }
 
@@ -544,8 +558,8 @@ cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, 
                                void* dX_e, float* dG, int64_t total, int d, cudaStream_t st) {
   const int qpr = d / 4;
   const unsigned grid = grid_for(total * 32, 256, 148 * 16);
-  if (dtype == 0) bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)dX_out, X_e, G, I, (float*)dX_e, dG, total, qpr);
-  else bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)dX_out, X_e, G, I, (bf16*)dX_e, dG, total, qpr);
+  if (dtype == 0) { count_launch(); bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)dX_out, X_e, G, I, (float*)dX_e, dG, total, qpr); }
+  else { count_launch(); bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)dX_out, X_e, G, I, (bf16*)dX_e, dG, total, qpr); }
   return cudaGetLastError();
 }
 
@@ -577,6 +591,7 @@ __global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __r
 
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr, const int32_t* slots,
                                float* dL, int64_t n, int E, int64_t k, cudaStream_t st) {
+  count_launch();
   bwd_softmax_kernel<<<grid_for(n * 32, 256, 148 * 16), 256, 0, st>>>(S, dG, row_ptr, slots, dL, n, E, k);
   return cudaGetLastError();
 }
@@ -594,8 +609,8 @@ __global__ void reduce_partials_kernel(const float* __restrict__ part, T* __rest
 }
 
 cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems, cudaStream_t st) {
-  if (dtype == 0) reduce_partials_kernel<float><<<grid_for(elems, 256), 256, 0, st>>>(part, (float*)out, P, elems);
-  else reduce_partials_kernel<bf16><<<grid_for(elems, 256), 256, 0, st>>>(part, (bf16*)out, P, elems);
+  if (dtype == 0) { count_launch(); reduce_partials_kernel<float><<<grid_for(elems, 256), 256, 0, st>>>(part, (float*)out, P, elems); }
+  else { count_launch(); reduce_partials_kernel<bf16><<<grid_for(elems, 256), 256, 0, st>>>(part, (bf16*)out, P, elems); }
   return cudaGetLastError();
 }
 
