@@ -3,14 +3,14 @@
 //
 //   C[b] (M x N, fp32 accumulate) = A[b] (M x K) . B[b] (K x N),  b = 0 .. batches-1
 //
-// One persistent CTA per SM, 192 threads, warp-specialised:
+// One persistent CTA per SM, 320 threads, warp-specialised:
 //   warp 0      TMA producer: fills a ring of shared-memory stages (A 128 x 64, B BN x 64 bf16,
 //               128-byte swizzle) with cp.async.bulk.tensor, one mbarrier per stage;
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M = 128, N = BN, K = 16) on shared-memory
 //               descriptors, accumulating in tensor memory; tcgen05.commit releases stages and
 //               publishes finished accumulators.  Two accumulators (2 x BN columns) are kept so the
 //               epilogue of one tile overlaps the main loop of the next;
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (one row of the tile per thread), apply the
+//   warps 2..9  epilogue (two per 32-lane quarter of tensor memory, half the columns each): tcgen05.ld the accumulator (one row of the tile per thread), apply the
 //               fused function (GeLU, GeLU', softmax), store.
 // Operands may be K-major (K contiguous in memory) or MN-major (M or N contiguous); the weights
 // W1, W2 [E, d, d'] and the activations are never transposed in memory, the shared-memory
@@ -31,7 +31,8 @@ namespace ecmoe {
 namespace {
 
 constexpr int BM = 128, BK = 64, UK = 16;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;                         // two per TMEM lane quarter, each takes half the columns
+constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;                 // 16 KiB
 constexpr int kSmemBudget = 200 * 1024;
 constexpr unsigned long long kWaitNs = 2000000000ull;
@@ -121,13 +122,28 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
          (1ull << 46) | (2ull << 61);
 }
 
-__device__ __forceinline__ float gelu_fwd(float z, int variant) {
-  if (variant == 0) return 0.5f * z * (1.f + erff(z * 0.70710678118654752f));
+// Phi(z) and exp(-z^2/2) with the rational approximation of erf of Abramowitz & Stegun 7.1.26
+// (|error| < 1.5e-7, far below bf16 resolution): erfc(x) = t(a1 + t(a2 + ... a5 t)) exp(-x^2),
+// t = 1/(1 + p x), x = |z|/sqrt(2).
+__device__ __forceinline__ float norm_cdf(float z, float& e) {
+  const float x = fabsf(z) * 0.70710678118654752f;
+  const float t = __fdividef(1.f, fmaf(0.3275911f, x, 1.f));
+  e = exp2f(-0.72134752044448170f * z * z);                   // exp(-z^2/2)
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float qq = 0.5f * poly * t * e;                       // 0.5 * erfc(x)
+  return z >= 0.f ? 1.f - qq : qq;
+}
+template <int VARIANT>
+__device__ __forceinline__ float gelu_fwd(float z) {
+  if (VARIANT == 0) { float e; return z * norm_cdf(z, e); }
   return 0.5f * z * (1.f + tanhf(0.7978845608028654f * (z + 0.044715f * z * z * z)));
 }
-__device__ __forceinline__ float gelu_bwd(float z, int variant) {
-  if (variant == 0)
-    return 0.5f * (1.f + erff(z * 0.70710678118654752f)) + z * 0.3989422804014327f * __expf(-0.5f * z * z);
+template <int VARIANT>
+__device__ __forceinline__ float gelu_bwd(float z) {
+  if (VARIANT == 0) { float e; const float Phi = norm_cdf(z, e); return fmaf(z * 0.3989422804014327f, e, Phi); }
   const float a = 0.7978845608028654f;
   const float th = tanhf(a * (z + 0.044715f * z * z * z));
   return 0.5f * (1.f + th) + 0.5f * z * (1.f - th * th) * a * (1.f + 3.f * 0.044715f * z * z);
@@ -159,7 +175,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 32 * kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -237,6 +253,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------------ epilogue, one tile row per thread
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;              // which half of the tile's columns this warp handles
+    constexpr int kHalf = BN / 2;
     int it = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++it) {
       const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
@@ -250,6 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int n0 = nt * BN;
       const int64_t obase = (int64_t)b * p.batch_c + (int64_t)row * p.ldc;
       if constexpr (EPI == EPI_SOFTMAX) {
+       if (half == 0) {                             // a row's softmax stays in one thread
         // Eq. 2: softmax over the N = E columns of this row; columns >= N are padding.
         float mx = -INFINITY;
         for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
@@ -278,8 +297,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
+       }
       } else {
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+#pragma unroll 1
+        for (int c0 = half * kHalf; c0 < (half + 1) * kHalf; c0 += 32) {
           if (n0 + c0 >= p.N) break;               // uniform across the warp
           uint32_t r[32]; tc_ld32(taddr + c0, r);
           if (!row_ok) continue;
@@ -308,7 +329,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               if (n0 + c0 + j < p.N) {
                 float z[8], h[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[j + e]); h[e] = gelu_fwd(z[e], p.gelu); }
+                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[j + e]); h[e] = p.gelu == 0 ? gelu_fwd<0>(z[e]) : gelu_fwd<1>(z[e]); }
                 *reinterpret_cast<uint4*>(p.C + o + j) = pack8(z);
                 *reinterpret_cast<uint4*>(p.C2 + o + j) = pack8(h);
               }
@@ -323,8 +344,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                   const float z0 = __uint_as_float(zw[e] << 16), z1 = __uint_as_float(zw[e] & 0xFFFF0000u);
-                  f[2 * e] = __uint_as_float(r[j + 2 * e]) * gelu_bwd(z0, p.gelu);
-                  f[2 * e + 1] = __uint_as_float(r[j + 2 * e + 1]) * gelu_bwd(z1, p.gelu);
+                  f[2 * e] = __uint_as_float(r[j + 2 * e]) * (p.gelu == 0 ? gelu_bwd<0>(z0) : gelu_bwd<1>(z0));
+                  f[2 * e + 1] = __uint_as_float(r[j + 2 * e + 1]) * (p.gelu == 0 ? gelu_bwd<0>(z1) : gelu_bwd<1>(z1));
                 }
                 *reinterpret_cast<uint4*>(p.C + o + j) = pack8(f);
               }
