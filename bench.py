@@ -32,6 +32,7 @@ WORKLOADS = {
     # name: (n, d, d', E, c)   shapes of Table 1 at sequence length 1024
     "cfg4": (16384, 4096, 16384, 64, 2.0),      # 8B/64E-shaped layer (headline)
     "cfg2": (8192, 768, 3072, 32, 2.0),         # 100M/32E-shaped layer
+    "cfg4e4": (1024, 4096, 16384, 4, 2.0),      # four experts of the 8B/64E shape (profiling-sized)
     "small": (2048, 256, 512, 8, 2.0),
 }
 GEMM_STAGES = ("gemm1_gelu", "gemm2", "gemm_dZ", "gemm_dW2", "gemm_dW1", "gemm_dXin")

@@ -34,7 +34,9 @@ constexpr int BM = 128, BK = 64, UK = 16;
 constexpr int kEpiWarps = 8;                         // two per TMEM lane quarter, each takes half the columns
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;                 // 16 KiB
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemBudget = 192 * 1024;              // operand stages; the epilogue's staging comes on top
+constexpr int kStagingPerWarp = 4096;
+constexpr int EPI_STORE_F32 = 5;                     // like EPI_STORE with fp32 output
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 __host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + bn * BK * 2; }
@@ -94,6 +96,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -160,14 +170,15 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // ---------------------------------------------------------------------------------------------
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmC2, const TcParams p) {
   constexpr int S = num_stages(BN);
   constexpr int kBBytes = BN * BK * 2;
   constexpr int kStage = kABytes + kBBytes;
   constexpr int kCols = tmem_cols(BN);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = (uint64_t*)(smem + S * kStage);          // full[S], empty[S], tmem_full[2], tmem_empty[2]
+  uint64_t* bars = (uint64_t*)(smem + S * kStage + kEpiWarps * kStagingPerWarp);   // full[S], empty[S], tmem_full[2], tmem_empty[2]
   uint32_t* tmem_slot = (uint32_t*)(bars + 2 * S + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, tfull0 = empty0 + 8 * S, tempty0 = tfull0 + 16;
@@ -299,56 +310,79 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
        }
       } else {
+        // Results leave through shared memory and the TMA unit: each warp converts a 32 x 32 chunk,
+        // writes it swizzled (conflict-free) into its own staging area and one lane issues a bulk
+        // tensor store, which writes whole lines and clips what overhangs M or N.
+        uint8_t* stg = smem + S * kStage + (warp - 2) * kStagingPerWarp;
+        const uint32_t stg_s = smem_u32(stg);
+        const int r0 = mt * BM + q * 32;
 #pragma unroll 1
         for (int c0 = half * kHalf; c0 < (half + 1) * kHalf; c0 += 32) {
           if (n0 + c0 >= p.N) break;               // uniform across the warp
           uint32_t r[32]; tc_ld32(taddr + c0, r);
-          if (!row_ok) continue;
-          const int64_t o = obase + n0 + c0;
-          if constexpr (EPI == EPI_STORE) {
-            if (p.Cf) {
+          if constexpr (EPI == EPI_STORE_F32) {
+            if (lane == 0) bulk_wait_read<0>();    // one 4 KiB buffer: 32 rows of 128 B, 128-byte swizzle
+            __syncwarp();
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                if (n0 + c0 + j < p.N)
-                  *reinterpret_cast<float4*>(p.Cf + o + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                         __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-            } else {
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                  make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s, n0 + c0, r0, b); bulk_commit(); }
+          } else {
+            // bf16: 32 rows of 64 B, 64-byte swizzle; two 2 KiB halves
+            const int sw = (lane >> 1) & 3;
+            if constexpr (EPI == EPI_GELU) {
+              if (lane == 0) bulk_wait_read<0>();
+              __syncwarp();
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                if (n0 + c0 + j < p.N) {
-                  float f[8];
-#pragma unroll
-                  for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[j + e]);
-                  *reinterpret_cast<uint4*>(p.C + o + j) = pack8(f);
-                }
-              }
-            }
-          } else if constexpr (EPI == EPI_GELU) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              if (n0 + c0 + j < p.N) {
+              for (int j = 0; j < 4; ++j) {
                 float z[8], h[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[j + e]); h[e] = p.gelu == 0 ? gelu_fwd<0>(z[e]) : gelu_fwd<1>(z[e]); }
-                *reinterpret_cast<uint4*>(p.C + o + j) = pack8(z);
-                *reinterpret_cast<uint4*>(p.C2 + o + j) = pack8(h);
+                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[8 * j + e]); h[e] = p.gelu == 0 ? gelu_fwd<0>(z[e]) : gelu_fwd<1>(z[e]); }
+                *reinterpret_cast<uint4*>(stg + lane * 64 + ((j ^ sw) << 4)) = pack8(z);
+                *reinterpret_cast<uint4*>(stg + 2048 + lane * 64 + ((j ^ sw) << 4)) = pack8(h);
               }
-            }
-          } else if constexpr (EPI == EPI_GELU_GRAD) {
+              fence_async_smem();
+              __syncwarp();
+              if (lane == 0 && r0 < p.M) {
+                tma_store_3d(&tmC, stg_s, n0 + c0, r0, b);
+                tma_store_3d(&tmC2, stg_s + 2048, n0 + c0, r0, b);
+                bulk_commit();
+              }
+            } else {
+              const int hb = ((c0 >> 5) & 1) * 2048;
+              float zf[32];
+              if constexpr (EPI == EPI_GELU_GRAD) {
+                const bf16* zp = p.Zin + obase + n0 + c0;
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              if (n0 + c0 + j < p.N) {
-                const uint4 zv = *reinterpret_cast<const uint4*>(p.Zin + o + j);
-                const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w};
+                for (int j = 0; j < 4; ++j) {
+                  uint4 zv = make_uint4(0, 0, 0, 0);
+                  if (row_ok && n0 + c0 + 8 * j < p.N) zv = *reinterpret_cast<const uint4*>(zp + 8 * j);
+                  const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    zf[8 * j + 2 * e] = __uint_as_float(zw[e] << 16);
+                    zf[8 * j + 2 * e + 1] = __uint_as_float(zw[e] & 0xFFFF0000u);
+                  }
+                }
+              }
+              if (lane == 0) bulk_wait_read<1>();  // the other half may still be in flight
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
                 float f[8];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  const float z0 = __uint_as_float(zw[e] << 16), z1 = __uint_as_float(zw[e] & 0xFFFF0000u);
-                  f[2 * e] = __uint_as_float(r[j + 2 * e]) * (p.gelu == 0 ? gelu_bwd<0>(z0) : gelu_bwd<1>(z0));
-                  f[2 * e + 1] = __uint_as_float(r[j + 2 * e + 1]) * (p.gelu == 0 ? gelu_bwd<0>(z1) : gelu_bwd<1>(z1));
+                for (int e = 0; e < 8; ++e) {
+                  f[e] = __uint_as_float(r[8 * j + e]);
+                  if constexpr (EPI == EPI_GELU_GRAD) f[e] *= p.gelu == 0 ? gelu_bwd<0>(zf[8 * j + e]) : gelu_bwd<1>(zf[8 * j + e]);
                 }
-                *reinterpret_cast<uint4*>(p.C + o + j) = pack8(f);
+                *reinterpret_cast<uint4*>(stg + hb + lane * 64 + ((j ^ sw) << 4)) = pack8(f);
               }
+              fence_async_smem();
+              __syncwarp();
+              if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + hb, n0 + c0, r0, b); bulk_commit(); }
             }
           }
         }
@@ -359,6 +393,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 
   // ------------------------------------------------------------------ orderly exit
+  if (warp >= 2 && lane == 0) bulk_wait_all();     // this warp's stores have left shared memory and are complete
   if (*abort_flag) {                               // let copies and MMAs still in flight drain
     const unsigned long long t0 = globaltimer();
     while (globaltimer() - t0 < 200000ull) __nanosleep(1000);
@@ -387,25 +422,27 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode() {
   return fn;
 }
 
-// Tensor map over a bf16 matrix stored [batches][rows][inner] with row pitch ld and batch pitch bs (elements).
+// Tensor map over a matrix stored [batches][rows][inner] with row pitch ld and batch pitch bs (elements).
 bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, int64_t batches, int64_t ld, int64_t bs,
-              int box_inner, int box_rows) {
+              int box_inner, int box_rows, bool f32 = false, CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
   auto enc = get_encode();
   if (!enc) return false;
+  const cuuint64_t es_bytes = f32 ? 4 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)batches};
-  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(batches > 1 ? bs : rows * ld) * 2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * es_bytes, (cuuint64_t)(batches > 1 ? bs : rows * ld) * es_bytes};
   cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
-  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  return enc(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
+             dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int pick_bn(const TcGemmArgs& g) { return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64); }
 
 template <int BN, int EPI>
-cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t st) {
-  constexpr int smem = num_stages(BN) * stage_bytes(BN) + 1024 + 256;
+cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                       const TcParams& p, cudaStream_t st) {
+  constexpr int smem = num_stages(BN) * stage_bytes(BN) + kEpiWarps * kStagingPerWarp + 1024 + 256;
   cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 148;
@@ -413,15 +450,16 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const TcPar
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
   count_launch();
-  gemm_tc_kernel<BN, EPI><<<grid, kThreads, smem, st>>>(ta, tb, p);
+  gemm_tc_kernel<BN, EPI><<<grid, kThreads, smem, st>>>(ta, tb, tc, tc2, p);
   return cudaGetLastError();
 }
 
 template <int EPI>
-cudaError_t launch_bn(int bn, const CUtensorMap& ta, const CUtensorMap& tb, const TcParams& p, cudaStream_t st) {
-  if (bn == 256) return launch_one<256, EPI>(ta, tb, p, st);
-  if (bn == 128) return launch_one<128, EPI>(ta, tb, p, st);
-  return launch_one<64, EPI>(ta, tb, p, st);
+cudaError_t launch_bn(int bn, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+                      const TcParams& p, cudaStream_t st) {
+  if (bn == 256) return launch_one<256, EPI>(ta, tb, tc, tc2, p, st);
+  if (bn == 128) return launch_one<128, EPI>(ta, tb, tc, tc2, p, st);
+  return launch_one<64, EPI>(ta, tb, tc, tc2, p, st);
 }
 
 }  // namespace
@@ -445,6 +483,14 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, g.K, g.batches, g.ldb, g.batch_b, 64, BK)
                                 : make_map(&tb, g.B, g.K, g.N, g.batches, g.ldb, g.batch_b, BK, bn);
   if (!oka || !okb) return cudaErrorInvalidValue;
+  // outputs leave through TMA stores of 32 x 32 chunks (64-byte rows for bf16, 128-byte rows for fp32)
+  CUtensorMap tc = ta, tc2 = ta;
+  if (g.epi != EPI_SOFTMAX) {
+    if (!make_map(&tc, g.C, g.N, g.M, g.batches, g.ldc, g.batch_c, 32, 32, g.c_f32 != 0,
+                  g.c_f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B)) return cudaErrorInvalidValue;
+    if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 32, 32, false,
+                                       CU_TENSOR_MAP_SWIZZLE_64B)) return cudaErrorInvalidValue;
+  }
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.batches = g.batches; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
   p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + bn - 1) / bn;
@@ -454,10 +500,11 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.C2 = (bf16*)g.C2; p.Zin = (const bf16*)g.Zin; p.S = g.S;
   p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
   switch (g.epi) {
-    case EPI_STORE: return launch_bn<EPI_STORE>(bn, ta, tb, p, st);
-    case EPI_GELU: return launch_bn<EPI_GELU>(bn, ta, tb, p, st);
-    case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ta, tb, p, st);
-    case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ta, tb, p, st);
+    case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ta, tb, tc, tc2, p, st)
+                                   : launch_bn<EPI_STORE>(bn, ta, tb, tc, tc2, p, st);
+    case EPI_GELU: return launch_bn<EPI_GELU>(bn, ta, tb, tc, tc2, p, st);
+    case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ta, tb, tc, tc2, p, st);
+    case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ta, tb, tc, tc2, p, st);
   }
   return cudaErrorInvalidValue;
 }
