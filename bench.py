@@ -60,7 +60,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -93,6 +93,12 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def workload_desc(name):
+    n, d, dff, E, c = WORKLOADS[name]
+    return (f"{name}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} fwd+bwd, bf16 storage / fp32 accumulate, "
+            f"one routing group per GPU")
+
+
 def layer_flops(n, d, dff, E, c):
     slots = int(n * c)
     gemm = 2.0 * slots * d * dff                 # one expert-batched GEMM
@@ -101,9 +107,10 @@ def layer_flops(n, d, dff, E, c):
 
 
 # ----------------------------------------------------------------------------------- CPU oracle timing
-def time_oracle_sample(n, d, dff, E, c, seed=0, experts=1):
-    """Times the oracle on routing in full plus `experts` whole experts forward + backward and
-    extrapolates the expert part to E experts.  Returns (tokens/s, threads, description)."""
+def time_oracle_sample(n, d, dff, E, c, seed=0, budget_s=12.0):
+    """Times the oracle on routing in full plus as many whole experts forward + backward as fit in
+    about `budget_s` seconds of CPU work (at least one, at most E) and extrapolates the expert part
+    to E experts.  Returns (tokens/s, threads, description)."""
     import numpy as np
     import torch
     from oracle import ec_oracle as O
@@ -118,22 +125,28 @@ def time_oracle_sample(n, d, dff, E, c, seed=0, experts=1):
     Wg = IN.normal_tensor((d, E), 1.0 / math.sqrt(d), seed, IN.TID_WG, bf).float().numpy().astype(np.float64)
     dY = IN.normal_tensor((n, d), 1.0, seed, IN.TID_DXOUT, bf).float().numpy().astype(np.float64)
     per = d * dff
-    W1 = [(IN.normal_chunk(seed, IN.TID_W1, i * per, per) / math.sqrt(d)).to(bf).float().numpy().astype(np.float64).reshape(d, dff)
-          for i in range(experts)]
-    W2 = [(IN.normal_chunk(seed, IN.TID_W2, i * per, per) / math.sqrt(dff)).to(bf).float().numpy().astype(np.float64).reshape(d, dff)
-          for i in range(experts)]
+
+    def weights(tid, i, fan_in):
+        w = (IN.normal_chunk(seed, tid, i * per, per) / math.sqrt(fan_in)).to(bf)
+        return w.float().numpy().astype(np.float64).reshape(d, dff)
+
     t0 = time.perf_counter()
     r = O.route(X, Wg, c)
     t_route = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    for i in range(experts):
+    t_sum, experts = 0.0, 0
+    while experts < E and (experts == 0 or t_route + t_sum < budget_s):
+        i = experts
+        W1_i, W2_i = weights(IN.TID_W1, i, d), weights(IN.TID_W2, i, dff)      # generation is not timed
+        t0 = time.perf_counter()
         I_i, G_i = r["I"][i], r["G"][i]
         X_in = X[I_i]
-        Z, H, X_e = O.expert_ffn(X_in, W1[i], W2[i])
+        Z, H, X_e = O.expert_ffn(X_in, W1_i, W2_i)
         dX_e = G_i[:, None] * dY[I_i]
         dG = np.einsum("jd,jd->j", dY[I_i], X_e)
-        O.expert_ffn_backward(dX_e, X_in, Z, H, W1[i], W2[i])
-    t_exp = (time.perf_counter() - t0) / experts
+        O.expert_ffn_backward(dX_e, X_in, Z, H, W1_i, W2_i)
+        t_sum += time.perf_counter() - t0
+        experts += 1
+    t_exp = t_sum / experts
     total = t_route + E * t_exp
     what = (f"oracle (numpy fp64) on n={n} d={d} d'={dff} E={E} c={c}: routing in full ({t_route:.2f} s) + "
             f"{experts} of {E} experts forward+backward ({t_exp:.2f} s each), expert part extrapolated x{E}; "
@@ -154,7 +167,7 @@ def run_reference(args):
     out = {"impl": "reference", "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": v, "unit": "tokens/s",
            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / v,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"{args.workload}: n={n} d={d} d_ff={dff} E={E} c={c}"},
+           "config": {"workload": workload_desc(args.workload)},
            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -278,8 +291,7 @@ def run_gpu(args):
             "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": world * n / (ms_step * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} "
-                                   f"fwd+bwd, bf16 storage / fp32 accumulate, one routing group per GPU",
+            "config": {"workload": workload_desc(args.workload),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
                              if args.workload != "small" else "small case, L2 resident",
                        "tensor_cores": bool(B.ec_uses_tensor_cores(cfg))},
@@ -305,7 +317,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
