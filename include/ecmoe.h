@@ -99,6 +99,45 @@ ec_status ec_route(const ec_config* cfg, const void* X, const void* Wg, float* S
                    void* cuda_stream);
 
 /*
+ * Routing for callers that cannot allocate device memory.  The paper has no counterpart:
+ * this is ec_route with the workspace argument taken away.
+ *
+ * Who needs it: code that is handed its input and output buffers by someone else and
+ * has no allocator of its own to ask for scratch, for example a plug-in running inside
+ * a host framework that owns all device memory, a real-time or serving loop in which
+ * cudaMalloc is forbidden because it synchronises the device and can fail or stall at
+ * an arbitrary moment, or a process whose memory budget was fixed at start-up.  Such a
+ * caller still passes X, Wg and the five outputs exactly as for ec_route; the scratch
+ * (status word, selection histograms and keys, inverse-index cursor) comes from a fixed
+ * array of EC_ROUTE_STATIC_SCRATCH_BYTES bytes that is part of the library's device
+ * image.  Every GPU on which the library is used holds that array from the moment the
+ * library's device code is loaded there until the process exits.
+ *
+ * Limits and behaviour
+ *  - A configuration whose routing scratch (ec_route_static_bytes(cfg)) exceeds
+ *    EC_ROUTE_STATIC_SCRATCH_BYTES is refused with EC_ERR_WORKSPACE and nothing is
+ *    launched; use ec_route with a workspace of your own for it.  8 MiB covers, for
+ *    instance, n = 262144 with E = 8 .. 256 at c = 2.
+ *  - The call itself makes no allocation: no cudaMalloc / cudaFree, no allocating
+ *    library routine.  The first call on each device looks up the array's device address
+ *    (once, with that device current, under a lock); make that first call outside any
+ *    stream capture.  Later calls on that device only queue work on `cuda_stream`.
+ *  - All calls on one device share the one array and it keeps the previous call's
+ *    contents; everything that must start at zero is cleared on `cuda_stream` at the
+ *    start of each call.  Two calls that can overlap on the GPU (different streams
+ *    without an ordering between them, or different host threads doing so) race on the
+ *    array and give undefined results: order them, or use ec_route with separate
+ *    workspaces.  There is no status word to read back afterwards; a caller that needs
+ *    ec_read_status uses ec_route.
+ *  - Results are those of ec_route on the same inputs, bit for bit.
+ */
+#define EC_ROUTE_STATIC_SCRATCH_BYTES (8u << 20)
+size_t ec_route_static_bytes(const ec_config* cfg); /* scratch this cfg needs; 0 on a bad cfg */
+ec_status ec_route_static(const ec_config* cfg, const void* X, const void* Wg, float* S,
+                          int32_t* I, float* G, int32_t* row_ptr, int32_t* slots,
+                          void* cuda_stream);
+
+/*
  * Forward, Eq. 2-4: routing as above, X_in = P . X (gather), X_e[i] =
  * GeLU(X_in[i] . W1[i]) . W2[i]^T for every expert, and X_out[t, :] = sum over the
  * slots (i, j) holding t of G[i, j] * X_e[i, j, :], experts in ascending order, in

@@ -21,7 +21,9 @@ EC_GELU_ERF, EC_GELU_TANH = 0, 1
 
 EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
-           "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read"]
+           "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
+           "ec_route_static", "ec_route_static_bytes"]
+EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class ec_config(C.Structure):
@@ -55,6 +57,9 @@ def lib():
         L.ec_saved_view.restype = C.c_int; L.ec_saved_view.argtypes = [P, V, C.POINTER(ec_saved_ptrs)]
         L.ec_route.restype = C.c_int
         L.ec_route.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V]
+        L.ec_route_static.restype = C.c_int
+        L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
+        L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
         L.ec_moe_forward.restype = C.c_int
         L.ec_moe_forward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, C.c_size_t, V]
         L.ec_moe_backward.restype = C.c_int
@@ -151,6 +156,20 @@ def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
     ws = alloc_workspace(cfg, dev) if ws is None else ws
     _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
                           _ptr(out.row_ptr), _ptr(out.slots), _ptr(ws), ws.numel(), _stream()), "ec_route")
+    return out
+
+
+def ec_route_static_bytes(cfg: ec_config) -> int:
+    return int(lib().ec_route_static_bytes(C.byref(cfg)))
+
+
+def ec_route_static(cfg, X, Wg, out: Routing) -> Routing:
+    """ec_route without a workspace: the scratch is a fixed array inside the library, for callers
+    that cannot allocate device memory.  `out` must be given (this call allocates nothing); calls
+    on one device must not overlap on the GPU.  Configurations that need more than
+    EC_ROUTE_STATIC_SCRATCH_BYTES of scratch raise EC_ERR_WORKSPACE."""
+    _check(lib().ec_route_static(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
+                                 _ptr(out.row_ptr), _ptr(out.slots), _stream()), "ec_route_static")
     return out
 
 

@@ -6,6 +6,7 @@
 #include <math.h>
 #include <string.h>
 #include <atomic>
+#include <mutex>
 
 using namespace ecmoe;
 
@@ -153,6 +154,33 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
   return EC_OK;
 }
 
+// Scratch of ec_route_static: lives in the library's own device image, so every GPU that loads
+// the library holds these bytes until the process exits.  The name below is only a handle on the
+// host; the device address is looked up once per device (static_scratch) and handed to the kernels.
+static __device__ __align__(256) unsigned char g_route_scratch[EC_ROUTE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_route_scratch on the current device; resolved on the first call per device.
+ec_status static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return EC_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_route_scratch) != cudaSuccess || !p) return EC_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  *out = g_static_ptr[dev];
+  return EC_OK;
+}
+
+// Bytes of scratch the routing stages alone use (the status word, the selection state and the
+// inverse-index cursor); the backward buffers that share the workspace are not part of it.
+size_t route_scratch_bytes(const Dims& D, const WsLayout& W) { return W.inverse + up(inverse_scratch_bytes(D.n)); }
+
 }  // namespace
 
 namespace ecmoe { void count_launch(int n) { g_launches += n; } }
@@ -195,6 +223,29 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   const WsLayout W = ws_layout(D);
   if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  prof_begin(st);
+  return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
+}
+
+size_t ec_route_static_bytes(const ec_config* c) {
+  Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
+  return route_scratch_bytes(D, ws_layout(D));
+}
+
+ec_status ec_route_static(const ec_config* c, const void* X, const void* Wg, float* S, int32_t* I, float* G,
+                          int32_t* row_ptr, int32_t* slots, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X || !Wg || !S || !I || !G || !row_ptr || !slots) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(S, 16) || misaligned(I, 16) || misaligned(G, 16) ||
+      misaligned(row_ptr, 16) || misaligned(slots, 16)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D);
+  if (route_scratch_bytes(D, W) > (size_t)EC_ROUTE_STATIC_SCRATCH_BYTES) return EC_ERR_WORKSPACE;
+  void* ws = nullptr;
+  if ((s = static_scratch(&ws)) != EC_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  // The array keeps whatever the previous call left: the status word is cleared here, and the
+  // routing stages clear their own counters, histograms and cursors before they use them.
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   prof_begin(st);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
