@@ -18,6 +18,17 @@
 // TMA unit zero-fill whatever a tile overhangs, so ragged M, N and K need no special code.
 // Tiles are ordered with M fastest so that CTAs running together share the same weight tile in L2.
 //
+// Two-CTA mode (CTAS = 2, used whenever M > 128): the two CTAs of a cluster work on one
+// 256 x BN tile.  Each loads its own 128 rows of A and its own half (BN / 2 rows) of B, so a
+// k-block costs each SM 32 KiB of fill instead of 48 KiB for the same 128 x 256 block of
+// accumulators; the main loop is bound by the L2 -> shared-memory fill rate, which is what
+// this buys.  Both producers announce their bytes on, and their copies complete on, the
+// full barrier of the even ("leader") CTA; the leader's thread issues tcgen05.mma.cta_group::2,
+// which reads both CTAs' shared memory and writes both CTAs' tensor memory (each keeps its own
+// 128 rows); tcgen05.commit with a two-CTA multicast releases the stage and publishes the
+// accumulator in both.  Each CTA's epilogue warps drain their own rows and report to the
+// leader's barrier.  Loads never use cluster multicast.
+//
 // Every wait on an mbarrier is bounded: after about two seconds the kernel records
 // EC_ERR_TIMEOUT in the status word, all roles leave their loops and the CTA exits in order.
 #include "internal.h"
@@ -25,6 +36,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <mutex>
+#include <string.h>
 
 namespace ecmoe {
 
@@ -39,9 +51,13 @@ constexpr int kStagingPerWarp = 4096;
 constexpr int EPI_STORE_F32 = 5;                     // like EPI_STORE with fp32 output
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
+// bn = rows of B one CTA loads per k-block (BN / CTAS)
 __host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + bn * BK * 2; }
 __host__ __device__ constexpr int num_stages(int bn) { return kSmemBudget / stage_bytes(bn) > 8 ? 8 : kSmemBudget / stage_bytes(bn); }
-__host__ __device__ constexpr int tmem_cols(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }   // power of two for bn = 64, 128, 256
+// Two accumulators of BN columns (a power of two for BN = 64, 128, 256).  A CTA pair takes all 512
+// columns, so both CTAs are certain to get base address 0: one tcgen05.mma writes the same
+// tensor-memory address in both.
+__host__ __device__ constexpr int tmem_cols(int bn, int ctas) { return ctas == 2 ? 512 : (2 * bn < 32 ? 32 : 2 * bn); }
 
 struct TcParams {
   int M, N, K, batches;
@@ -95,6 +111,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// Two-CTA forms.  The barrier operands are shared::cluster addresses (possibly the peer's).
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {   // arrives on the barrier at this offset in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
@@ -168,14 +207,16 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmC2, const TcParams p) {
-  constexpr int S = num_stages(BN);
-  constexpr int kBBytes = BN * BK * 2;
+  constexpr int BNL = BN / CTAS;                    // rows of B this CTA loads
+  constexpr int TM = BM * CTAS;                     // rows of the tile the CTA (pair) works on
+  constexpr int S = num_stages(BNL);
+  constexpr int kBBytes = BNL * BK * 2;
   constexpr int kStage = kABytes + kBBytes;
-  constexpr int kCols = tmem_cols(BN);
+  constexpr int kCols = tmem_cols(BN, CTAS);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = (uint64_t*)(smem + S * kStage + kEpiWarps * kStagingPerWarp);   // full[S], empty[S], tmem_full[2], tmem_empty[2]
@@ -183,10 +224,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, tfull0 = empty0 + 8 * S, tempty0 = tfull0 + 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;      // 0 = leader of the pair
+  const int first_tile = blockIdx.x / CTAS, tile_step = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
+    // full: one arrival, the (leader's) producer announcing the bytes of the whole pair; tmem_empty: one per epilogue warp of the pair
     for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, 32 * kEpiWarps); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, CTAS * kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -196,51 +240,79 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (CTAS == 2) cluster_sync_all();     // the peer's barriers exist before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t smem_base = smem_u32(smem);
   bool gave_up = false;
+  if (CTAS == 2 && tmem_base != 0) {               // cannot happen with all 512 columns taken; refuse rather than corrupt
+    if (threadIdx.x == 0) { atomicExch(p.status + 1, 9); atomicExch(p.status, 5); }
+    gave_up = true;
+  }
 
-  if (warp == 0) {
+  if (gave_up) {
+    // nothing: fall through to the exit sequence
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles && !gave_up; tile += gridDim.x) {
+      const uint32_t leader_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
+      for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step) {
         const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
-        const int m0 = mt * BM, n0 = nt * BN;
+        const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
-          const uint32_t bar = full0 + 8 * stage;
           const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
-          mbar_expect_tx(bar, kStage);
           const int k0 = kb * BK;
-          if (p.a_mn) {                       // stored [K][M]: boxes of 64 (M) x 64 (K)
+          if constexpr (CTAS == 2) {
+            // The leader's barrier collects both halves: its producer announces the pair's bytes, the
+            // peer's copies simply complete on it (they may land before the announcement; the phase
+            // cannot end before the leader's arrival and a byte count of zero).
+            const uint32_t bar = leader_full0 + 8 * stage;
+            if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * kStage);
+            if (p.a_mn) {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
-          } else {                            // stored [M][K]: one box 64 (K) x 128 (M)
-            tma_load_3d(sa, &tmA, bar, k0, m0, b);
-          }
-          if (p.b_mn) {
+              for (int j = 0; j < BM / 64; ++j) tma_load_3d_pair(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
+            } else {
+              tma_load_3d_pair(sa, &tmA, bar, k0, m0, b);
+            }
+            if (p.b_mn) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+              for (int j = 0; j < BNL / 64; ++j) tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+            } else {
+              tma_load_3d_pair(sb, &tmB, bar, k0, n0, b);
+            }
           } else {
-            tma_load_3d(sb, &tmB, bar, k0, n0, b);
+            const uint32_t bar = full0 + 8 * stage;
+            mbar_expect_tx(bar, kStage);
+            if (p.a_mn) {                       // stored [K][M]: boxes of 64 (M) x 64 (K)
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
+            } else {                            // stored [M][K]: one box 64 (K) x 128 (M)
+              tma_load_3d(sa, &tmA, bar, k0, m0, b);
+            }
+            if (p.b_mn) {
+#pragma unroll
+              for (int j = 0; j < BNL / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+            } else {
+              tma_load_3d(sb, &tmB, bar, k0, n0, b);
+            }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (the leader's, in a pair)
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
       // K-major: 8-row groups 1024 B apart, 32 B per K step inside the swizzle atom.
       // MN-major: 64-wide blocks BK*128 B apart (LBO), 8-row K groups 1024 B apart (SBO), 2 groups per K step.
       const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
       const uint32_t a_step = p.a_mn ? 2048 : 32, b_step = p.b_mn ? 2048 : 32;
       int stage = 0; uint32_t phase = 0; int it = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles && !gave_up; tile += gridDim.x, ++it) {
+      for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step, ++it) {
         const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
         if (!mbar_wait(tempty0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.status, 2)) { gave_up = true; break; }
         tc_fence_after();
@@ -253,12 +325,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int kk = 0; kk < BK / UK; ++kk) {
             const uint64_t ad = make_desc(sa + kk * a_step, a_lbo, 1024);
             const uint64_t bd = make_desc(sb + kk * b_step, b_lbo, 1024);
-            tc_mma(d_tmem, ad, bd, idesc, (kb | kk) != 0);
+            if constexpr (CTAS == 2) tc_mma_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0);
+            else tc_mma(d_tmem, ad, bd, idesc, (kb | kk) != 0);
           }
-          tc_commit(empty0 + 8 * stage);           // stage is free once these MMAs have read it
+          // the stage is free (in both CTAs) once these MMAs have read it
+          if constexpr (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
           if (++stage == S) { stage = 0; phase ^= 1; }
         }
-        if (!gave_up) tc_commit(tfull0 + 8 * buf); // accumulator complete
+        if (!gave_up) {                              // accumulator complete
+          if constexpr (CTAS == 2) tc_commit_pair(tfull0 + 8 * buf); else tc_commit(tfull0 + 8 * buf);
+        }
       }
     }
   } else {
@@ -267,13 +343,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;              // which half of the tile's columns this warp handles
     constexpr int kHalf = BN / 2;
     int it = 0;
-    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x, ++it) {
+    const uint32_t tempty_leader = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
+    for (int tile = first_tile; tile < p.total_tiles; tile += tile_step, ++it) {
       const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
       const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
       const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
       tc_fence_after();
-      const int row = mt * BM + q * 32 + lane;
+      const int row = mt * TM + (int)rank * BM + q * 32 + lane;
       const bool row_ok = row < p.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * BN;
       const int n0 = nt * BN;
@@ -315,7 +392,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // tensor store, which writes whole lines and clips what overhangs M or N.
         uint8_t* stg = smem + S * kStage + (warp - 2) * kStagingPerWarp;
         const uint32_t stg_s = smem_u32(stg);
-        const int r0 = mt * BM + q * 32;
+        const int r0 = mt * TM + (int)rank * BM + q * 32;
 #pragma unroll 1
         for (int c0 = half * kHalf; c0 < (half + 1) * kHalf; c0 += 32) {
           if (n0 + c0 >= p.N) break;               // uniform across the warp
@@ -388,7 +465,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       tc_fence_before();
-      mbar_arrive(tempty0 + 8 * buf);              // 128 arrivals free the accumulator
+      __syncwarp();                                // every lane's tcgen05.ld has completed
+      if (lane == 0) {                             // one arrival per warp frees the accumulator
+        if constexpr (CTAS == 2) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(tempty0 + 8 * buf);
+      }
     }
   }
 
@@ -401,6 +481,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncwarp();
   tc_fence_before();
   __syncthreads();
+  if constexpr (CTAS == 2) cluster_sync_all();     // the peer no longer reads this CTA's shared or writes its tensor memory
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kCols) : "memory");
@@ -438,28 +519,55 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
 }
 
 int pick_bn(const TcGemmArgs& g) { return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64); }
+// Two CTAs per tile when a tile of 256 rows is not mostly padding and the pair's B halves are whole 64-wide blocks.
+int pick_ctas(const TcGemmArgs& g, int bn) { return (g.epi != EPI_SOFTMAX && bn >= 128 && g.M > BM) ? 2 : 1; }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                        const TcParams& p, cudaStream_t st) {
-  constexpr int smem = num_stages(BN) * stage_bytes(BN) + kEpiWarps * kStagingPerWarp + 1024 + 256;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  constexpr int smem = num_stages(BN / CTAS) * stage_bytes(BN / CTAS) + kEpiWarps * kStagingPerWarp + 1024 + 256;
+  auto kern = gemm_tc_kernel<BN, EPI, CTAS>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  cudaLaunchConfig_t cfg; memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  int groups = sms / CTAS;                           // CTAs (or pairs) that run at once
+  if (CTAS == 2) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    static int max_pairs[64] = {};                   // pairs the device can hold at once, per device
+    if (dev >= 0 && dev < 64) {
+      if (max_pairs[dev] == 0) {
+        cfg.gridDim = dim3(2 * groups);
+        int nc = 0;
+        if (cudaOccupancyMaxActiveClusters(&nc, kern, &cfg) == cudaSuccess && nc > 0) max_pairs[dev] = nc; else max_pairs[dev] = groups;
+      }
+      if (max_pairs[dev] < groups) groups = max_pairs[dev];
+    }
+  }
+  if (p.total_tiles < groups) groups = p.total_tiles;
+  cfg.gridDim = dim3(groups * CTAS);
   count_launch();
-  gemm_tc_kernel<BN, EPI><<<grid, kThreads, smem, st>>>(ta, tb, tc, tc2, p);
-  return cudaGetLastError();
+  return cudaLaunchKernelEx(&cfg, kern, ta, tb, tc, tc2, p);
 }
 
 template <int EPI>
-cudaError_t launch_bn(int bn, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
+cudaError_t launch_bn(int bn, int ctas, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                       const TcParams& p, cudaStream_t st) {
-  if (bn == 256) return launch_one<256, EPI>(ta, tb, tc, tc2, p, st);
-  if (bn == 128) return launch_one<128, EPI>(ta, tb, tc, tc2, p, st);
-  return launch_one<64, EPI>(ta, tb, tc, tc2, p, st);
+  if constexpr (EPI != EPI_SOFTMAX) {
+    if (ctas == 2) {
+      if (bn == 256) return launch_one<256, EPI, 2>(ta, tb, tc, tc2, p, st);
+      return launch_one<128, EPI, 2>(ta, tb, tc, tc2, p, st);
+    }
+  }
+  if (bn == 256) return launch_one<256, EPI, 1>(ta, tb, tc, tc2, p, st);
+  if (bn == 128) return launch_one<128, EPI, 1>(ta, tb, tc, tc2, p, st);
+  return launch_one<64, EPI, 1>(ta, tb, tc, tc2, p, st);
 }
 
 }  // namespace
@@ -476,12 +584,14 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
 
 cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   const int bn = pick_bn(g);
+  const int ctas = pick_ctas(g, bn);
+  const int bnl = bn / ctas;                         // rows of B one CTA loads
   CUtensorMap ta, tb;
   // A: K-major [M rows][K inner], box 64 x 128;  MN-major [K rows][M inner], box 64 x 64
   const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, g.K, g.batches, g.lda, g.batch_a, 64, BK)
                                 : make_map(&ta, g.A, g.K, g.M, g.batches, g.lda, g.batch_a, BK, BM);
   const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, g.K, g.batches, g.ldb, g.batch_b, 64, BK)
-                                : make_map(&tb, g.B, g.K, g.N, g.batches, g.ldb, g.batch_b, BK, bn);
+                                : make_map(&tb, g.B, g.K, g.N, g.batches, g.ldb, g.batch_b, BK, bnl);
   if (!oka || !okb) return cudaErrorInvalidValue;
   // outputs leave through TMA stores of 32 x 32 chunks (64-byte rows for bf16, 128-byte rows for fp32)
   CUtensorMap tc = ta, tc2 = ta;
@@ -493,18 +603,18 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   }
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.batches = g.batches; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
-  p.tiles_m = (g.M + BM - 1) / BM; p.tiles_n = (g.N + bn - 1) / bn;
+  p.tiles_m = (g.M + BM * ctas - 1) / (BM * ctas); p.tiles_n = (g.N + bn - 1) / bn;
   p.total_tiles = p.tiles_m * p.tiles_n * g.batches; p.kblocks = (g.K + BK - 1) / BK;
   p.gelu = g.gelu;
   p.C = g.c_f32 ? nullptr : (bf16*)g.C; p.Cf = g.c_f32 ? (float*)g.C : nullptr;
   p.C2 = (bf16*)g.C2; p.Zin = (const bf16*)g.Zin; p.S = g.S;
   p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
   switch (g.epi) {
-    case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ta, tb, tc, tc2, p, st)
-                                   : launch_bn<EPI_STORE>(bn, ta, tb, tc, tc2, p, st);
-    case EPI_GELU: return launch_bn<EPI_GELU>(bn, ta, tb, tc, tc2, p, st);
-    case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ta, tb, tc, tc2, p, st);
-    case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ta, tb, tc, tc2, p, st);
+    case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
+                                   : launch_bn<EPI_STORE>(bn, ctas, ta, tb, tc, tc2, p, st);
+    case EPI_GELU: return launch_bn<EPI_GELU>(bn, ctas, ta, tb, tc, tc2, p, st);
+    case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ctas, ta, tb, tc, tc2, p, st);
+    case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ctas, ta, tb, tc, tc2, p, st);
   }
   return cudaErrorInvalidValue;
 }
