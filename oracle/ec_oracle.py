@@ -202,7 +202,7 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     dS = np.zeros((n, e), F64)
     for i in range(e):
         dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
-    dL = S * (dS - (dS * S).sum(axis=1, keepdims=True))    # softmax Jacobian, per token row
+    dL = store("dL", S * (dS - (dS * S).sum(axis=1, keepdims=True)))   # softmax Jacobian, per token row
     dWg = store("dWg", X.T @ dL)
     dX = dL @ Wg.T
     for i in range(e):

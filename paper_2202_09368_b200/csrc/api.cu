@@ -52,7 +52,15 @@ SavedLayout saved_layout(const Dims& D) {
   return L;
 }
 
-int dwg_splits(const Dims& D) { int64_t p = (D.n + 1023) / 1024; return (int)(p < 1 ? 1 : (p > 32 ? 32 : p)); }
+// Number of fixed cuts of the token axis in dWg = X^T . dL: enough (row tile, cut) pairs for about two
+// waves of CTAs, at least 512 tokens per cut, at most 32 cuts.  Depends on the shape only, so the
+// summation order, and with it the result, is the same on every run.
+int dwg_splits(const Dims& D) {
+  const int64_t tiles_m = (D.d + 127) / 128;
+  int64_t p = 296 / tiles_m;
+  if (p > D.n / 512) p = D.n / 512;
+  return (int)(p < 1 ? 1 : (p > 32 ? 32 : p));
+}
 
 struct WsLayout { size_t status, topk, inverse, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
 WsLayout ws_layout(const Dims& D) {
@@ -301,7 +309,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   const int32_t* row_ptr = (const int32_t*)(sv + L.row_ptr); const int32_t* slots = (const int32_t*)(sv + L.slots);
   const void* X_in = sv + L.X_in; const void* Z = sv + L.Z; const void* H = sv + L.H; const float* X_e = (const float*)(sv + L.X_e);
   void* dX_e = w + W.dX_e; float* dG = (float*)(w + W.dG); void* dZ = w + W.dZ; void* dX_in = w + W.dX_in;
-  float* dL = (float*)(w + W.dL); float* part = (float*)(w + W.dWg_part);
+  void* dL = w + W.dL; float* part = (float*)(w + W.dWg_part);
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
@@ -325,12 +333,31 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
   if ((s = run_gemm(D, g6, status, st)) != EC_OK) return s;
   prof_mark("gemm_dXin", st);
-  // softmax backward: dL [n, E] fp32
-  EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, D.n, D.E, D.k, st));
+  // softmax backward: dL [n, E]; bf16 when the two gate-gradient products below run on tensor cores
+  const int P = dwg_splits(D);
+  TcGemmArgs tw; memset(&tw, 0, sizeof(tw));          // dWg = X^T . dL, cut along the tokens
+  const int64_t cut = (((D.n + P - 1) / P) + 63) / 64 * 64;
+  tw.A = X; tw.a_mn_major = 1; tw.lda = D.d; tw.B = dL; tw.b_mn_major = 1; tw.ldb = D.E;
+  tw.M = D.d; tw.N = D.E; tw.K = (int)cut; tw.batches = P; tw.k_split = 1; tw.k_total = D.n;
+  tw.epi = EPI_STORE; tw.c_f32 = 1; tw.C = part; tw.ldc = D.E; tw.batch_c = (int64_t)D.d * D.E; tw.status = status;
+  TcGemmArgs tx; memset(&tx, 0, sizeof(tx));          // dX = dL . Wg^T + rows of dX_in
+  tx.A = dL; tx.a_mn_major = 0; tx.lda = D.E; tx.B = Wg; tx.b_mn_major = 0; tx.ldb = D.E;
+  tx.M = (int)D.n; tx.N = D.d; tx.K = D.E; tx.batches = 1;
+  tx.epi = EPI_ADD_SLOTS; tx.C = dX; tx.ldc = D.d; tx.status = status;
+  tx.row_ptr = row_ptr; tx.slots = slots; tx.rows = dX_in; tx.ld_rows = D.d;
+  const bool tc_gate = D.dtype == EC_BF16 && tc_gemm_supported(tw) && tc_gemm_supported(tx);
+  EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, tc_gate ? 1 : 0, D.n, D.E, D.k, st));
   prof_mark("bwd_softmax", st);
+  if (tc_gate) {
+    EC_CUDA(launch_gemm_tc(tw, st));
+    EC_CUDA(launch_reduce_partials(D.dtype, part, dWg, P, (int64_t)D.d * D.E, st));
+    prof_mark("dWg", st);
+    EC_CUDA(launch_gemm_tc(tx, st));
+    prof_mark("dX", st);
+    return EC_OK;
+  }
   // dWg = X^T . dL, split over the tokens into fixed chunks and summed in a fixed order
   {
-    const int P = dwg_splits(D);
     const int64_t chunk = (D.n + P - 1) / P;
     GemmArgs g; memset(&g, 0, sizeof(g));
     g.A = X; g.B = dL; g.C = part; g.a_dtype = D.dtype; g.b_dtype = EC_F32; g.c_dtype = EC_F32;

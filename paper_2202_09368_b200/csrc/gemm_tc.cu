@@ -67,6 +67,8 @@ struct TcParams {
   bf16* C; bf16* C2; const bf16* Zin; float* Cf; float* S;
   int64_t ldc, batch_c;
   int* status;
+  int k_split;                                       // batches are cuts of one product along K
+  const int32_t* row_ptr; const int32_t* slots; const bf16* rows; int64_t ld_rows;   // EPI_ADD_SLOTS
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -263,7 +265,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
           const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
-          const int k0 = kb * BK;
+          const int k0 = kb * BK + (p.k_split ? b * p.K : 0);
+          const int bc = p.k_split ? 0 : b;          // third coordinate of the operand maps
           if constexpr (CTAS == 2) {
             // The leader's barrier collects both halves: its producer announces the pair's bytes, the
             // peer's copies simply complete on it (they may land before the announcement; the phase
@@ -272,30 +275,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * kStage);
             if (p.a_mn) {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j) tma_load_3d_pair(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
+              for (int j = 0; j < BM / 64; ++j) tma_load_3d_pair(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, bc);
             } else {
-              tma_load_3d_pair(sa, &tmA, bar, k0, m0, b);
+              tma_load_3d_pair(sa, &tmA, bar, k0, m0, bc);
             }
             if (p.b_mn) {
 #pragma unroll
-              for (int j = 0; j < BNL / 64; ++j) tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+              for (int j = 0; j < BNL / 64; ++j) tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, bc);
             } else {
-              tma_load_3d_pair(sb, &tmB, bar, k0, n0, b);
+              tma_load_3d_pair(sb, &tmB, bar, k0, n0, bc);
             }
           } else {
             const uint32_t bar = full0 + 8 * stage;
             mbar_expect_tx(bar, kStage);
             if (p.a_mn) {                       // stored [K][M]: boxes of 64 (M) x 64 (K)
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, b);
+              for (int j = 0; j < BM / 64; ++j) tma_load_3d(sa + j * (BK * 128), &tmA, bar, m0 + 64 * j, k0, bc);
             } else {                            // stored [M][K]: one box 64 (K) x 128 (M)
-              tma_load_3d(sa, &tmA, bar, k0, m0, b);
+              tma_load_3d(sa, &tmA, bar, k0, m0, bc);
             }
             if (p.b_mn) {
 #pragma unroll
-              for (int j = 0; j < BNL / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+              for (int j = 0; j < BNL / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, bc);
             } else {
-              tma_load_3d(sb, &tmB, bar, k0, n0, b);
+              tma_load_3d(sb, &tmB, bar, k0, n0, bc);
             }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
@@ -445,6 +448,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   }
                 }
               }
+              if constexpr (EPI == EPI_ADD_SLOTS) {
+                // this thread's row gains the rows of its slots (64 bytes of each), in slot order
+                if (row_ok) {
+                  const int qa = p.row_ptr[row], qb = p.row_ptr[row + 1];
+                  for (int qq = qa; qq < qb; ++qq) {
+                    const bf16* src = p.rows + (int64_t)p.slots[qq] * p.ld_rows + n0 + c0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                      if (n0 + c0 + 8 * j < p.N) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + 8 * j);
+                        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                          r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) + __uint_as_float(w[e] << 16));
+                          r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) + __uint_as_float(w[e] & 0xFFFF0000u));
+                        }
+                      }
+                    }
+                  }
+                }
+              }
               if (lane == 0) bulk_wait_read<1>();  // the other half may still be in flight
               __syncwarp();
 #pragma unroll
@@ -578,6 +602,9 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
   if (g.batches > 1 && (g.batch_a % 8 || g.batch_b % 8 || g.batch_c % 8)) return false;
   if (((uintptr_t)g.A | (uintptr_t)g.B) & 15) return false;
   if (g.epi == EPI_SOFTMAX && (g.N > 256 || g.batches != 1)) return false;
+  if (g.k_split && (g.K % BK || g.k_total < 1 || !g.c_f32 || g.epi != EPI_STORE)) return false;
+  if (g.epi == EPI_ADD_SLOTS && (g.batches != 1 || g.c_f32 || !g.row_ptr || !g.slots || !g.rows || g.ld_rows % 8 ||
+                                 ((uintptr_t)g.rows & 15))) return false;
   if ((int64_t)g.lda * 2 >= ((int64_t)1 << 40) || (int64_t)g.ldb * 2 >= ((int64_t)1 << 40)) return false;
   return true;
 }
@@ -588,10 +615,13 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   const int bnl = bn / ctas;                         // rows of B one CTA loads
   CUtensorMap ta, tb;
   // A: K-major [M rows][K inner], box 64 x 128;  MN-major [K rows][M inner], box 64 x 64
-  const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, g.K, g.batches, g.lda, g.batch_a, 64, BK)
-                                : make_map(&ta, g.A, g.K, g.M, g.batches, g.lda, g.batch_a, BK, BM);
-  const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, g.K, g.batches, g.ldb, g.batch_b, 64, BK)
-                                : make_map(&tb, g.B, g.K, g.N, g.batches, g.ldb, g.batch_b, BK, bnl);
+  // operand maps: with k_split both are single matrices whose K extent is the whole contraction
+  const int64_t kext = g.k_split ? g.k_total : g.K;
+  const int64_t ob = g.k_split ? 1 : g.batches;
+  const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, kext, ob, g.lda, g.batch_a, 64, BK)
+                                : make_map(&ta, g.A, kext, g.M, ob, g.lda, g.batch_a, BK, BM);
+  const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, kext, ob, g.ldb, g.batch_b, 64, BK)
+                                : make_map(&tb, g.B, kext, g.N, ob, g.ldb, g.batch_b, BK, bnl);
   if (!oka || !okb) return cudaErrorInvalidValue;
   // outputs leave through TMA stores of 32 x 32 chunks (64-byte rows for bf16, 128-byte rows for fp32)
   CUtensorMap tc = ta, tc2 = ta;
@@ -609,11 +639,14 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.C = g.c_f32 ? nullptr : (bf16*)g.C; p.Cf = g.c_f32 ? (float*)g.C : nullptr;
   p.C2 = (bf16*)g.C2; p.Zin = (const bf16*)g.Zin; p.S = g.S;
   p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
+  p.k_split = g.k_split;
+  p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows;
   switch (g.epi) {
     case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
                                    : launch_bn<EPI_STORE>(bn, ctas, ta, tb, tc, tc2, p, st);
     case EPI_GELU: return launch_bn<EPI_GELU>(bn, ctas, ta, tb, tc, tc2, p, st);
     case EPI_GELU_GRAD: return launch_bn<EPI_GELU_GRAD>(bn, ctas, ta, tb, tc, tc2, p, st);
+    case EPI_ADD_SLOTS: return launch_bn<EPI_ADD_SLOTS>(bn, ctas, ta, tb, tc, tc2, p, st);
     case EPI_SOFTMAX: return launch_bn<EPI_SOFTMAX>(bn, ctas, ta, tb, tc, tc2, p, st);
   }
   return cudaErrorInvalidValue;

@@ -42,9 +42,10 @@ cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const in
 cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, const float* G,
                                const int32_t* I, void* dX_e, float* dG, int64_t slots_total, int d,
                                cudaStream_t st);
-// dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] S[t,i']),  dS scattered from dG through the inverse index
+// dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] S[t,i']),  dS scattered from dG through the inverse index;
+// dL is stored as bf16 when dl_bf16 (operand of the tensor-core dWg / dX products), else fp32
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr,
-                               const int32_t* slots, float* dL, int64_t n, int E, int64_t k,
+                               const int32_t* slots, void* dL, int dl_bf16, int64_t n, int E, int64_t k,
                                cudaStream_t st);
 // out[r,c] = sum_p part[p,r,c] in ascending p (fixed order), cast to dtype
 cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems,
@@ -81,6 +82,13 @@ struct TcGemmArgs {
   int c_f32;
   float* S;         // EPI_SOFTMAX: fp32 row softmax of the N columns, [M, N]
   int* status;      // device status word
+  // k_split != 0: one matrix product cut along K.  A and B are single matrices (batch strides unused),
+  // `batches` is the number of cuts and K the length of one (a multiple of 64); cut b contracts rows
+  // b*K .. b*K+K-1 (those at or beyond k_total count as zero) and writes the partial result C[b] (fp32).
+  int k_split; int64_t k_total;
+  // EPI_ADD_SLOTS (bf16 C, batches == 1): C[m, :] = acc[m, :] + sum over q in [row_ptr[m], row_ptr[m+1]) of
+  // rows[slots[q], :] in ascending q, summed in fp32 and rounded once.
+  const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;
 };
 constexpr int EPI_SOFTMAX = 4;
 bool tc_gemm_supported(const TcGemmArgs& g);

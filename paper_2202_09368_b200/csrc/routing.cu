@@ -567,9 +567,13 @@ cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, 
 // Backward of the softmax of Eq. 2, one warp per token.  dS[t,i] is dG of the slot of expert i that
 // holds t (0 if none);  dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] * S[t,i']).
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void st_dl(float* p, int64_t i, float v) { p[i] = v; }
+__device__ __forceinline__ void st_dl(bf16* p, int64_t i, float v) { p[i] = __float2bfloat16(v); }
+
+template <typename TL>
 __global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __restrict__ dG,
                                    const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
-                                   float* __restrict__ dL, int64_t n, int E, int64_t k) {
+                                   TL* __restrict__ dL, int64_t n, int E, int64_t k) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < n; t += warps) {
@@ -580,19 +584,21 @@ __global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __r
       dot = fmaf(dG[s], S[t * E + s / k], dot);
     }
     for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    for (int i = lane; i < E; i += 32) dL[t * E + i] = -S[t * E + i] * dot;
+    for (int i = lane; i < E; i += 32) st_dl(dL, t * E + i, -S[t * E + i] * dot);
     __syncwarp();
     for (int q = a + lane; q < b; q += 32) {           // the slots of one token belong to distinct experts
       const int s = slots[q]; const int64_t i = s / k;
-      dL[t * E + i] = S[t * E + i] * (dG[s] - dot);
+      st_dl(dL, t * E + i, S[t * E + i] * (dG[s] - dot));
     }
   }
 }
 
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr, const int32_t* slots,
-                               float* dL, int64_t n, int E, int64_t k, cudaStream_t st) {
+                               void* dL, int dl_bf16, int64_t n, int E, int64_t k, cudaStream_t st) {
   count_launch();
-  bwd_softmax_kernel<<<grid_for(n * 32, 256, 148 * 16), 256, 0, st>>>(S, dG, row_ptr, slots, dL, n, E, k);
+  const unsigned grid = grid_for(n * 32, 256, 148 * 16);
+  if (dl_bf16) bwd_softmax_kernel<bf16><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (bf16*)dL, n, E, k);
+  else bwd_softmax_kernel<float><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (float*)dL, n, E, k);
   return cudaGetLastError();
 }
 

@@ -9,7 +9,7 @@ compare it with the CPU oracle following the protocol
 
 Error measure: max|gpu - ref| / RMS(ref), per tensor.  Bound: 1e-4 on the fp32 path.
 On the bf16 path the bound is 2e-2, except where the storage format alone already
-costs more: the layer keeps Z, H, dX_e, dZ, dX_in and its outputs in bf16 (they
+costs more: the layer keeps Z, H, dX_e, dZ, dX_in, dL and its outputs in bf16 (they
 are tensor-core operands or bf16 activations by definition of the path), and its
 outputs are heavy-tailed (a token's row scales with its gate weights), so the
 exact fp64 result rounded once to bf16 can sit above 2e-2 by itself.  The test
@@ -33,7 +33,7 @@ def rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / rms)
 
 
-BF16_STORED = {"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dX", "dWg", "dW1", "dW2"}
+BF16_STORED = {"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2"}
 
 
 def bf16_store(name, x):
