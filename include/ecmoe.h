@@ -185,10 +185,13 @@ long long ec_launch_count(void);
  * Per-stage device timing, for benchmarks (no counterpart in the paper).  After
  * ec_profile_enable(1), each call of ec_route / ec_moe_forward / ec_moe_backward records a CUDA
  * event on its stream after every stage (gate, top-k, inverse index, gather, the GEMMs, combine,
- * ...).  ec_profile_read waits for the last call's final event and writes up to max_stages
- * elapsed times (milliseconds) and static stage names in launch order; it returns the number of
- * stages, 0 when profiling is off, -1 on a CUDA error.  The state is global to the process: use
- * it from one thread, one call at a time.  Off by default.
+ * ...).  The events of the last routing / forward call and of the last backward call are kept
+ * apart, so a forward and a backward queued back to back can both be read afterwards.
+ * ec_profile_read waits for those calls' final events and writes up to max_stages elapsed times
+ * (milliseconds) and static stage names, forward stages first, then backward; it returns the
+ * number of stages written (what it returned is not returned again), 0 when profiling is off or
+ * nothing was recorded, -1 on a CUDA error.  The state is global to the process: use it from one
+ * thread, one call of each kind at a time.  Off by default.
  */
 void ec_profile_enable(int on);
 int ec_profile_read(float* ms, const char** names, int max_stages);

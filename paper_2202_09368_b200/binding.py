@@ -209,8 +209,8 @@ def ec_profile_enable(on: bool) -> None:
     lib().ec_profile_enable(1 if on else 0)
 
 
-def ec_profile_read(max_stages: int = 20):
-    """[(stage name, milliseconds), ...] of the last profiled call."""
+def ec_profile_read(max_stages: int = 40):
+    """[(stage name, milliseconds), ...] of the last profiled forward and backward calls."""
     ms = (C.c_float * max_stages)()
     names = (C.c_char_p * max_stages)()
     cnt = lib().ec_profile_read(ms, names, max_stages)

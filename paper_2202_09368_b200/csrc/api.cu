@@ -87,28 +87,34 @@ inline bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)
 #define EC_CUDA(x) do { if ((x) != cudaSuccess) return EC_ERR_CUDA; } while (0)
 
 // Optional per-stage timing (ec_profile_enable): an event is recorded on the call's stream after
-// each stage of forward / backward.  Host state only; off by default and then free of cost.
+// each stage.  Two sets of events, one for routing / forward calls and one for backward calls, so
+// that a forward + backward pair queued back to back can be read afterwards without a
+// synchronisation in between.  Host state only; off by default and then free of cost.
 constexpr int kMaxStages = 20;
 struct Profile {
-  bool enabled = false;
   cudaEvent_t ev[kMaxStages + 1];
   bool created = false;
-  int count = 0;                       // stages recorded by the last call
+  int count = 0;                       // stages recorded by the last call of this kind
   const char* names[kMaxStages];
 };
-Profile g_prof;
+bool g_prof_enabled = false;
+Profile g_prof[2];
+int g_prof_cur = 0;
 std::atomic<long long> g_launches{0};
 
-void prof_begin(cudaStream_t st) {
-  if (!g_prof.enabled) return;
-  if (!g_prof.created) { for (auto& e : g_prof.ev) cudaEventCreate(&e); g_prof.created = true; }
-  g_prof.count = 0;
-  cudaEventRecord(g_prof.ev[0], st);
+void prof_begin(cudaStream_t st, int kind) {
+  if (!g_prof_enabled) return;
+  Profile& P = g_prof[kind];
+  g_prof_cur = kind;
+  if (!P.created) { for (auto& e : P.ev) cudaEventCreate(&e); P.created = true; }
+  P.count = 0;
+  cudaEventRecord(P.ev[0], st);
 }
 void prof_mark(const char* name, cudaStream_t st) {
-  if (!g_prof.enabled || g_prof.count >= kMaxStages) return;
-  g_prof.names[g_prof.count] = name;
-  cudaEventRecord(g_prof.ev[++g_prof.count], st);
+  Profile& P = g_prof[g_prof_cur];
+  if (!g_prof_enabled || P.count >= kMaxStages) return;
+  P.names[P.count] = name;
+  cudaEventRecord(P.ev[++P.count], st);
 }
 
 // One expert-batched GEMM: tensor cores when the shape allows, FMA otherwise.
@@ -232,7 +238,7 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
-  prof_begin(st);
+  prof_begin(st, 0);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
 }
 
@@ -255,7 +261,7 @@ ec_status ec_route_static(const ec_config* c, const void* X, const void* Wg, flo
   // The array keeps whatever the previous call left: the status word is cleared here, and the
   // routing stages clear their own counters, histograms and cursors before they use them.
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
-  prof_begin(st);
+  prof_begin(st, 0);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
 }
 
@@ -274,7 +280,7 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; float* X_e = (float*)(sv + L.X_e);
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
-  prof_begin(st);
+  prof_begin(st, 0);
   if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st)) != EC_OK) return s;
   EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
   prof_mark("gather", st);
@@ -314,7 +320,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Eq. 4 backward: dX_e, dG
-  prof_begin(st);
+  prof_begin(st, 1);
   EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
   prof_mark("bwd_combine", st);
   // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
@@ -404,17 +410,22 @@ const char* ec_status_string(ec_status s) {
 
 long long ec_launch_count(void) { return g_launches.load(); }
 
-void ec_profile_enable(int on) { g_prof.enabled = on != 0; if (!on) g_prof.count = 0; }
+void ec_profile_enable(int on) { g_prof_enabled = on != 0; g_prof[0].count = g_prof[1].count = 0; }
 
 int ec_profile_read(float* ms, const char** names, int max_stages) {
-  if (!g_prof.enabled || g_prof.count == 0) return 0;
-  if (cudaEventSynchronize(g_prof.ev[g_prof.count]) != cudaSuccess) return -1;
-  int nst = g_prof.count < max_stages ? g_prof.count : max_stages;
-  for (int i = 0; i < nst; ++i) {
-    float t = 0.f;
-    if (cudaEventElapsedTime(&t, g_prof.ev[i], g_prof.ev[i + 1]) != cudaSuccess) return -1;
-    if (ms) ms[i] = t;
-    if (names) names[i] = g_prof.names[i];
+  if (!g_prof_enabled) return 0;
+  int nst = 0;
+  for (int kind = 0; kind < 2; ++kind) {
+    Profile& P = g_prof[kind];
+    if (P.count == 0) continue;
+    if (cudaEventSynchronize(P.ev[P.count]) != cudaSuccess) return -1;
+    for (int i = 0; i < P.count && nst < max_stages; ++i, ++nst) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, P.ev[i], P.ev[i + 1]) != cudaSuccess) return -1;
+      if (ms) ms[nst] = t;
+      if (names) names[nst] = P.names[i];
+    }
+    P.count = 0;
   }
   return nst;
 }

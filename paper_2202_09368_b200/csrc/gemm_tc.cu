@@ -16,7 +16,8 @@
 // W1, W2 [E, d, d'] and the activations are never transposed in memory, the shared-memory
 // descriptors carry the orientation.  Three-dimensional tensor maps (inner, rows, batch) let the
 // TMA unit zero-fill whatever a tile overhangs, so ragged M, N and K need no special code.
-// Tiles are ordered with M fastest so that CTAs running together share the same weight tile in L2.
+// Tiles are ordered with M fastest so that CTAs running together share the same weight tile in L2
+// (with N fastest for the weight gradients, whose output dominates: see launch_gemm_tc).
 //
 // Two-CTA mode (CTAS = 2, used whenever M > 128): the two CTAs of a cluster work on one
 // 256 x BN tile.  Each loads its own 128 rows of A and its own half (BN / 2 rows) of B, so a
@@ -46,8 +47,8 @@ constexpr int BM = 128, BK = 64, UK = 16;
 constexpr int kEpiWarps = 8;                         // two per TMEM lane quarter, each takes half the columns
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;                 // 16 KiB
-constexpr int kSmemBudget = 192 * 1024;              // operand stages; the epilogue's staging comes on top
-constexpr int kStagingPerWarp = 4096;
+constexpr int kSmemBudget = 160 * 1024;              // operand stages; the epilogue's staging comes on top
+constexpr int kStagingPerWarp = 8192;                // two 4 KiB buffers of 32 rows x 128 bytes
 constexpr int EPI_STORE_F32 = 5;                     // like EPI_STORE with fp32 output
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
@@ -63,6 +64,7 @@ struct TcParams {
   int M, N, K, batches;
   int a_mn, b_mn;
   int tiles_m, tiles_n, total_tiles, kblocks;
+  int n_fast;                                        // consecutive tiles run along N (else along M)
   int gelu;
   bf16* C; bf16* C2; const bf16* Zin; float* Cf; float* S;
   int64_t ldc, batch_c;
@@ -167,6 +169,20 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// The same load without the wait, so that several can be in flight; tc_ld_wait() completes them all.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
@@ -260,7 +276,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0; uint32_t phase = 0;
       const uint32_t leader_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
       for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step) {
-        const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
+        const int b = tile / (p.tiles_m * p.tiles_n);
+        const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
+        const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
         const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
@@ -344,11 +362,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ epilogue, one tile row per thread
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;              // which half of the tile's columns this warp handles
-    constexpr int kHalf = BN / 2;
     int it = 0;
+    uint32_t nchunk = 0;                           // chunks this warp has stored so far: picks the staging buffer
     const uint32_t tempty_leader = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
     for (int tile = first_tile; tile < p.total_tiles; tile += tile_step, ++it) {
-      const int mt = tile % p.tiles_m, nt = (tile / p.tiles_m) % p.tiles_n, b = tile / (p.tiles_m * p.tiles_n);
+      const int b = tile / (p.tiles_m * p.tiles_n);
+        const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
+        const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
       const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
       const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
@@ -390,72 +410,86 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
        }
       } else {
-        // Results leave through shared memory and the TMA unit: each warp converts a 32 x 32 chunk,
-        // writes it swizzled (conflict-free) into its own staging area and one lane issues a bulk
-        // tensor store, which writes whole lines and clips what overhangs M or N.
+        // Results leave through shared memory and the TMA unit.  A warp owns 32 rows and kColsPerWarp columns
+        // of the tile and works on chunks whose rows are 128 bytes long (64 bf16 or 32 fp32 columns): each
+        // thread converts its row of the chunk and writes it with the 128-byte swizzle (conflict-free) into one
+        // of the warp's two 4 KiB staging buffers, one lane issues a bulk tensor store, which writes whole
+        // 128-byte lines and clips what overhangs M or N.  The buffers alternate from chunk to chunk (across
+        // tiles too); one is reused once the store issued two chunks earlier has read it.
         uint8_t* stg = smem + S * kStage + (warp - 2) * kStagingPerWarp;
         const uint32_t stg_s = smem_u32(stg);
         const int r0 = mt * TM + (int)rank * BM + q * 32;
+        const int sw = lane & 7;
+        constexpr int kColsPerWarp = BN >= 128 ? BN / 2 : BN;      // a 64-wide tile is drained by the first four warps alone
+        const bool active = half * kColsPerWarp < BN;
+        if constexpr (EPI == EPI_STORE_F32) {
 #pragma unroll 1
-        for (int c0 = half * kHalf; c0 < (half + 1) * kHalf; c0 += 32) {
-          if (n0 + c0 >= p.N) break;               // uniform across the warp
-          uint32_t r[32]; tc_ld32(taddr + c0, r);
-          if constexpr (EPI == EPI_STORE_F32) {
-            if (lane == 0) bulk_wait_read<0>();    // one 4 KiB buffer: 32 rows of 128 B, 128-byte swizzle
+          for (int c0 = half * kColsPerWarp; active && c0 < (half + 1) * kColsPerWarp; c0 += 32, ++nchunk) {
+            if (n0 + c0 >= p.N) break;             // uniform across the warp
+            uint32_t r[32]; tc_ld32(taddr + c0, r);
+            uint8_t* bufp = stg + (nchunk & 1) * 4096;
+            if (lane == 0) bulk_wait_read<1>();
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+              *reinterpret_cast<uint4*>(bufp + lane * 128 + ((j ^ sw) << 4)) =
                   make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
             fence_async_smem();
             __syncwarp();
-            if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s, n0 + c0, r0, b); bulk_commit(); }
-          } else {
-            // bf16: 32 rows of 64 B, 64-byte swizzle; two 2 KiB halves
-            const int sw = (lane >> 1) & 3;
+            if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + (nchunk & 1) * 4096, n0 + c0, r0, b); bulk_commit(); }
+          }
+        } else {
+#pragma unroll 1
+          for (int c0 = half * kColsPerWarp; active && c0 < (half + 1) * kColsPerWarp; c0 += 64, ++nchunk) {
+            if (n0 + c0 >= p.N) break;             // uniform across the warp
+            uint32_t r[64];
+            tc_ld32_issue(taddr + c0, r); tc_ld32_issue(taddr + c0 + 32, r + 32); tc_ld_wait();
             if constexpr (EPI == EPI_GELU) {
+              // both buffers are written: Z into the first, H = GeLU(Z) into the second
               if (lane == 0) bulk_wait_read<0>();
               __syncwarp();
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
+              for (int j = 0; j < 8; ++j) {
                 float z[8], h[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[8 * j + e]); h[e] = p.gelu == 0 ? gelu_fwd<0>(z[e]) : gelu_fwd<1>(z[e]); }
-                *reinterpret_cast<uint4*>(stg + lane * 64 + ((j ^ sw) << 4)) = pack8(z);
-                *reinterpret_cast<uint4*>(stg + 2048 + lane * 64 + ((j ^ sw) << 4)) = pack8(h);
+                *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ sw) << 4)) = pack8(z);
+                *reinterpret_cast<uint4*>(stg + 4096 + lane * 128 + ((j ^ sw) << 4)) = pack8(h);
               }
               fence_async_smem();
               __syncwarp();
               if (lane == 0 && r0 < p.M) {
                 tma_store_3d(&tmC, stg_s, n0 + c0, r0, b);
-                tma_store_3d(&tmC2, stg_s + 2048, n0 + c0, r0, b);
+                tma_store_3d(&tmC2, stg_s + 4096, n0 + c0, r0, b);
                 bulk_commit();
               }
             } else {
-              const int hb = ((c0 >> 5) & 1) * 2048;
-              float zf[32];
               if constexpr (EPI == EPI_GELU_GRAD) {
+                // dZ = acc * GeLU'(Z): this thread's 64 values of Z (128 bytes of its row)
                 const bf16* zp = p.Zin + obase + n0 + c0;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < 8; ++j) {
                   uint4 zv = make_uint4(0, 0, 0, 0);
                   if (row_ok && n0 + c0 + 8 * j < p.N) zv = *reinterpret_cast<const uint4*>(zp + 8 * j);
                   const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w};
 #pragma unroll
                   for (int e = 0; e < 4; ++e) {
-                    zf[8 * j + 2 * e] = __uint_as_float(zw[e] << 16);
-                    zf[8 * j + 2 * e + 1] = __uint_as_float(zw[e] & 0xFFFF0000u);
+                    const float z0 = __uint_as_float(zw[e] << 16), z1 = __uint_as_float(zw[e] & 0xFFFF0000u);
+                    const float g0 = p.gelu == 0 ? gelu_bwd<0>(z0) : gelu_bwd<1>(z0);
+                    const float g1 = p.gelu == 0 ? gelu_bwd<0>(z1) : gelu_bwd<1>(z1);
+                    r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) * g0);
+                    r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) * g1);
                   }
                 }
               }
               if constexpr (EPI == EPI_ADD_SLOTS) {
-                // this thread's row gains the rows of its slots (64 bytes of each), in slot order
+                // this thread's row gains the rows of its slots (128 bytes of each), in slot order
                 if (row_ok) {
                   const int qa = p.row_ptr[row], qb = p.row_ptr[row + 1];
                   for (int qq = qa; qq < qb; ++qq) {
                     const bf16* src = p.rows + (int64_t)p.slots[qq] * p.ld_rows + n0 + c0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
+                    for (int j = 0; j < 8; ++j) {
                       if (n0 + c0 + 8 * j < p.N) {
                         const uint4 v = *reinterpret_cast<const uint4*>(src + 8 * j);
                         const unsigned w[4] = {v.x, v.y, v.z, v.w};
@@ -469,21 +503,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   }
                 }
               }
-              if (lane == 0) bulk_wait_read<1>();  // the other half may still be in flight
+              uint8_t* bufp = stg + (nchunk & 1) * 4096;
+              if (lane == 0) bulk_wait_read<1>();  // the other buffer's store may still be in flight
               __syncwarp();
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
+              for (int j = 0; j < 8; ++j) {
                 float f[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  f[e] = __uint_as_float(r[8 * j + e]);
-                  if constexpr (EPI == EPI_GELU_GRAD) f[e] *= p.gelu == 0 ? gelu_bwd<0>(zf[8 * j + e]) : gelu_bwd<1>(zf[8 * j + e]);
-                }
-                *reinterpret_cast<uint4*>(stg + hb + lane * 64 + ((j ^ sw) << 4)) = pack8(f);
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * j + e]);
+                *reinterpret_cast<uint4*>(bufp + lane * 128 + ((j ^ sw) << 4)) = pack8(f);
               }
               fence_async_smem();
               __syncwarp();
-              if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + hb, n0 + c0, r0, b); bulk_commit(); }
+              if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + (nchunk & 1) * 4096, n0 + c0, r0, b); bulk_commit(); }
             }
           }
         }
@@ -623,13 +655,11 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, kext, ob, g.ldb, g.batch_b, 64, BK)
                                 : make_map(&tb, g.B, kext, g.N, ob, g.ldb, g.batch_b, BK, bnl);
   if (!oka || !okb) return cudaErrorInvalidValue;
-  // outputs leave through TMA stores of 32 x 32 chunks (64-byte rows for bf16, 128-byte rows for fp32)
+  // outputs leave through TMA stores of chunks of 32 rows x 128 bytes (64 bf16 or 32 fp32 columns)
   CUtensorMap tc = ta, tc2 = ta;
   if (g.epi != EPI_SOFTMAX) {
-    if (!make_map(&tc, g.C, g.N, g.M, g.batches, g.ldc, g.batch_c, 32, 32, g.c_f32 != 0,
-                  g.c_f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B)) return cudaErrorInvalidValue;
-    if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 32, 32, false,
-                                       CU_TENSOR_MAP_SWIZZLE_64B)) return cudaErrorInvalidValue;
+    if (!make_map(&tc, g.C, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, 32, g.c_f32 != 0)) return cudaErrorInvalidValue;
+    if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 64, 32)) return cudaErrorInvalidValue;
   }
   TcParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.batches = g.batches; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
@@ -640,6 +670,11 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.C2 = (bf16*)g.C2; p.Zin = (const bf16*)g.Zin; p.S = g.S;
   p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
   p.k_split = g.k_split;
+  // Tile order.  Tiles running at the same time are consecutive ones.  Along M (default) they share the B tile,
+  // which for the expert FFNs is the weight matrix: it is then read from HBM once.  When the output is larger
+  // than the operands (short K: the weight gradients) the tiles run along N instead, so that what is written at
+  // one time is whole rows of C rather than 512-byte pieces 2*N bytes apart, and they share the A tile.
+  p.n_fast = (int64_t)g.M * g.N > ((int64_t)g.M + g.N) * g.K ? 1 : 0;
   p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows;
   switch (g.epi) {
     case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
