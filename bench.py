@@ -1,6 +1,7 @@
 """Benchmark of the expert-choice MoE layer (forward + backward) on B200.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4|cfg2|small] [--impl reference]
+  python bench.py --routing [--route-case n,E]      (routing-only stress, one extra JSON line format)
 
 A step is one forward + backward pass of the whole layer over one group of n tokens
 (routing, gather, expert FFNs, combine, and every backward kernel).  Prints ONE JSON
@@ -314,6 +315,77 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------------- routing-only stress
+ROUTING_GRID = [(n, E) for n in (4096, 16384, 65536, 262144) for E in (8, 32, 128, 256)]
+
+
+def routing_bytes(n, d, E, c, b=2):
+    """Algorithmic bytes each routing stage has to move (reads + writes), per call."""
+    slots = int(n * c)
+    return {
+        "gate_softmax": n * d * b + d * E * b + n * E * 4,
+        "topk": n * E * 4 + slots * 8,
+        "inverse_index": slots * 4 + (n + 1 + slots) * 4,
+        "gather": 2 * slots * d * b + slots * 4,
+        "combine": slots * d * 4 + slots * 4 + (n + 1 + slots) * 4 + n * d * b,
+    }
+
+
+def run_routing(args):
+    """Routing-only stress: gate + softmax, column top-k, inverse index, shuffle and unshuffle with
+    identity experts (X_e = X_in), d = 1024, bf16, c = 2.  Per stage: device time from the library's
+    stage events and algorithmic GB/s.  L2 is flushed (a 512 MiB buffer is overwritten) before every
+    timed call, so the small cases are not timed out of cache."""
+    import torch
+    from paper_2202_09368_b200 import binding as B
+    from paper_2202_09368_b200 import inputs as IN
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dev = torch.device("cuda")
+    d, c, bf = 1024, 2.0, torch.bfloat16
+    grid = ROUTING_GRID if not args.route_case else [tuple(int(v) for v in args.route_case.split(","))]
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    peaks = measured_peaks()
+    cases = []
+    B.ec_profile_enable(True)
+    for n, E in grid:
+        cfg = B.make_config(n, d, 8, E, c, bf)
+        X = IN.normal_tensor((n, d), 1.0, 0, IN.TID_X, bf, dev, 1 << 26)
+        Wg = IN.normal_tensor((d, E), 1.0 / math.sqrt(d), 0, IN.TID_WG, bf, dev, 1 << 26)
+        ws = B.alloc_workspace(cfg, dev)
+        r = B.ec_route(cfg, X, Wg, ws=ws)
+        X_in = B.ec_shuffle(cfg, X, r.I)
+        X_e = X_in.float()
+        X_out = torch.empty_like(X)
+        acc = {}
+        reps = max(3, min(args.steps, 20))
+        for it in range(3 + reps):
+            for call in (lambda: B.ec_route(cfg, X, Wg, ws=ws, out=r), lambda: B.ec_shuffle(cfg, X, r.I, X_in),
+                         lambda: B.ec_unshuffle(cfg, X_e, r.G, r.row_ptr, r.slots, X_out)):
+                flush.zero_()
+                call()
+                for k_, v_ in B.ec_profile_read():
+                    if it >= 3:
+                        acc.setdefault(k_, []).append(v_)
+        assert B.ec_read_status(ws) == B.EC_OK
+        by = routing_bytes(n, d, E, c)
+        st = {}
+        for k_, v_ in acc.items():
+            v_.sort()
+            med = v_[len(v_) // 2]
+            st[k_] = {"us": round(med * 1e3, 2), "GBps": round(by[k_] / (med * 1e-3) / 1e9, 1),
+                      "frac_hbm": round(by[k_] / (med * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+        total_us = sum(v["us"] for v in st.values())
+        cases.append({"n": n, "E": E, "k": int(n * c / E), "stages": st, "chain_us": round(total_us, 2),
+                      "chain_GBps": round(sum(by.values()) / (total_us * 1e-6) / 1e9, 1),
+                      "tokens_per_s": round(n / (total_us * 1e-6))})
+        del X, Wg, ws, r, X_in, X_e, X_out
+    B.ec_profile_enable(False)
+    print(json.dumps({"metric": "ec_routing_chain", "unit": "GB/s (algorithmic bytes / device time per stage)",
+                      "config": {"workload": "routing-only stress: d=1024 bf16 c=2, identity experts",
+                                 "l2": "512 MiB flush before every timed call"},
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cases": cases}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -322,8 +394,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
+    ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' instead of the grid")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.routing:
+        run_routing(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

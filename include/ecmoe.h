@@ -99,6 +99,24 @@ ec_status ec_route(const ec_config* cfg, const void* X, const void* Wg, float* S
                    void* cuda_stream);
 
 /*
+ * The shuffle of Eq. 3 on its own: X_in[i, j, :] = X[I[i, j], :] (X_in = P . X with P = Onehot(I)),
+ * a row gather.  X [n, d] and I [E, k] in, X_in [E, k, d] out, both of cfg->dtype.  Entries of I
+ * must lie in [0, n).  No workspace.
+ */
+ec_status ec_shuffle(const ec_config* cfg, const void* X, const int32_t* I, void* X_in,
+                     void* cuda_stream);
+
+/*
+ * The unshuffle of Eq. 4 on its own: X_out[t, :] = sum over the slots s = (i, j) that hold token t of
+ * G[s] * X_e[s, :], slots in ascending order, accumulated in fp32 and rounded once; rows of
+ * tokens without a slot are zero.  X_e [E, k, d] fp32, G [E, k] fp32 and the token -> slot index
+ * (row_ptr [n+1], slots [E*k], as ec_route writes them) in, X_out [n, d] of cfg->dtype out.
+ * No workspace, no atomics: the result does not depend on scheduling.
+ */
+ec_status ec_unshuffle(const ec_config* cfg, const float* X_e, const float* G, const int32_t* row_ptr,
+                       const int32_t* slots, void* X_out, void* cuda_stream);
+
+/*
  * Routing for callers that cannot allocate device memory.  The paper has no counterpart:
  * this is ec_route with the workspace argument taken away.
  *

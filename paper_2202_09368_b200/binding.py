@@ -22,7 +22,7 @@ EC_GELU_ERF, EC_GELU_TANH = 0, 1
 EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
-           "ec_route_static", "ec_route_static_bytes"]
+           "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle"]
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -60,6 +60,8 @@ def lib():
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
+        L.ec_shuffle.restype = C.c_int; L.ec_shuffle.argtypes = [P, V, V, V, V]
+        L.ec_unshuffle.restype = C.c_int; L.ec_unshuffle.argtypes = [P, V, V, V, V, V, V]
         L.ec_moe_forward.restype = C.c_int
         L.ec_moe_forward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, C.c_size_t, V]
         L.ec_moe_backward.restype = C.c_int
@@ -157,6 +159,24 @@ def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
     _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
                           _ptr(out.row_ptr), _ptr(out.slots), _ptr(ws), ws.numel(), _stream()), "ec_route")
     return out
+
+
+def ec_shuffle(cfg, X, I, X_in=None):
+    """Eq. 3 shuffle: X_in[i, j, :] = X[I[i, j], :]."""
+    k = ec_capacity(cfg)
+    if X_in is None:
+        X_in = torch.empty(cfg.E, k, cfg.d_model, dtype=X.dtype, device=X.device)
+    _check(lib().ec_shuffle(C.byref(cfg), _ptr(X), _ptr(I), _ptr(X_in), _stream()), "ec_shuffle")
+    return X_in
+
+
+def ec_unshuffle(cfg, X_e, G, row_ptr, slots, X_out=None):
+    """Eq. 4 unshuffle: X_out[t, :] = sum over the slots of t of G[s] * X_e[s, :] (X_e, G fp32)."""
+    if X_out is None:
+        X_out = torch.empty(cfg.n, cfg.d_model, dtype=_torch_dtype(cfg), device=X_e.device)
+    _check(lib().ec_unshuffle(C.byref(cfg), _ptr(X_e), _ptr(G), _ptr(row_ptr), _ptr(slots), _ptr(X_out), _stream()),
+           "ec_unshuffle")
+    return X_out
 
 
 def ec_route_static_bytes(cfg: ec_config) -> int:

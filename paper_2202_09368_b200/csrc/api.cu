@@ -242,6 +242,30 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
 }
 
+ec_status ec_shuffle(const ec_config* c, const void* X, const int32_t* I, void* X_in, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X || !I || !X_in) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(I, 16) || misaligned(X_in, 16)) return EC_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  prof_begin(st, 0);
+  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
+  prof_mark("gather", st);
+  return EC_OK;
+}
+
+ec_status ec_unshuffle(const ec_config* c, const float* X_e, const float* G, const int32_t* row_ptr,
+                       const int32_t* slots, void* X_out, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!X_e || !G || !row_ptr || !slots || !X_out) return EC_ERR_INVALID_ARG;
+  if (misaligned(X_e, 16) || misaligned(G, 16) || misaligned(row_ptr, 16) || misaligned(slots, 16) ||
+      misaligned(X_out, 16)) return EC_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  prof_begin(st, 0);
+  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
+  prof_mark("combine", st);
+  return EC_OK;
+}
+
 size_t ec_route_static_bytes(const ec_config* c) {
   Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
   return route_scratch_bytes(D, ws_layout(D));

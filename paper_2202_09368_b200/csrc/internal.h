@@ -11,14 +11,19 @@ namespace ecmoe {
 using bf16 = __nv_bfloat16;
 
 constexpr int kTopkChunk = 32;     // experts per histogram CTA column chunk
-constexpr int kRadixPasses = 8;    // 8-bit digits of the 64-bit (score, token) key
+constexpr int kRadixBits = 10;     // digit width of the radix selection
+constexpr int kRadixPasses = 3;    // the 30 significant bits of a score in (0, 1]
+constexpr int kCandCap = 512;      // threshold-bucket keys per expert the final sort may choose from
 constexpr int kSortTile = 4096;    // 64-bit keys sorted in shared memory by one CTA
 
 // Word 0 of the workspace: status written by kernels (0 = fine, 5 = a bounded wait expired).
 struct StatusWord { int code; int where; int pad[62]; };
 
 // Per-expert state of the radix selection.
-struct SelState { unsigned long long prefix; unsigned int k_rem; unsigned int done; };
+// prefix: key bits decided so far (bits below `shift` are open); k_rem: keys still wanted from the
+// threshold bucket; mode: 0 undecided, 1 take the whole bucket, 2 choose k_rem of `cand` candidates,
+// 3 ties at the threshold were taken in token order.
+struct SelState { unsigned long long prefix; unsigned int k_rem, mode, shift, cand; unsigned int pad[2]; };
 
 // ---- bookkeeping (api.cu) ----------------------------------------------------------------------
 // Every kernel launch of the library goes through count_launch(); ec_launch_count() reports the sum.

@@ -125,29 +125,36 @@ cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, f
 // ------------------------------------------------------------------------------------------
 // Column top-k, Eq. 2: G, I = TopK(S^T, k).
 //
-// Every (token t, expert i) entry gets the 64-bit key  (~bits(S[t,i]) << 32) | t.  S >= 0, so its
-// bit pattern is monotone in its value: a smaller key is a larger score, and among equal scores a
-// lower token.  Keys of one expert are distinct, so "the k smallest keys, ascending" is the
-// unique answer with ties broken toward the lower token and slots listed by descending score.
+// Every (token t, expert i) entry gets the 64-bit key  (~bits(S[t,i]) << 32) | t.  0 <= S <= 1, so its
+// bit pattern is below 2^30 and monotone in its value: a smaller key is a larger score, and among
+// equal scores a lower token.  Keys of one expert are distinct, so "the k smallest keys, ascending"
+// is the unique answer with ties broken toward the lower token and slots listed by descending score.
 //
-// Selection is a most-significant-digit radix select run for all experts at once: pass p
-// histograms digit p (8 bits) of the keys that still match the expert's prefix; the last CTA of a
-// column chunk to finish picks the digit in which the k-th key lies.  An expert is finished as
-// soon as the bucket it descends into holds exactly the number of keys still wanted (with
-// distinct scores that is after the four score digits; the token digits only run for ties at
-// the threshold).  Then one pass copies the keys not above the threshold and a bitonic network
-// sorts the k keys of each expert.
+// Selection is a most-significant-digit radix select over the 30 significant score bits, 10 bits a
+// pass, run for all experts at once: a pass histograms its digit of the keys that still match the
+// expert's prefix (in shared memory, merged into one global histogram per expert), and the last
+// CTA of a column chunk to finish picks the bucket in which the k-th key lies.  An expert leaves
+// the passes as soon as that bucket is small: either it holds exactly the keys still wanted, or at
+// most kCandCap keys, the candidates, from which the final sort picks the best.  With distinct
+// scores that is after two passes over S.  Experts still undecided after the three score passes
+// have more than kCandCap exactly equal scores at the threshold: there the lowest tokens win, and
+// one CTA per such expert walks the column in token order and takes the first ones.  One more pass
+// over S then copies the winners (and candidates) out, and a bitonic network sorts each expert's keys.
 //
-// scratch: [SelState E][hist passes*E*256 u32][counters passes*chunks u32][cursor E u32][keys E*kpad u64]
+// scratch: [SelState E][hist E*1024 u32][counters passes*chunks u32][cursors 2E u32] (zeroed per call)
+//          [candidates E*kCandCap u64][keys E*kpad u64]
 // ------------------------------------------------------------------------------------------
-constexpr int kHistThreads = 256;
+constexpr int kHistThreads = 1024;
+constexpr int kBins = 1 << kRadixBits;
+constexpr int kHistSmemBytes = (kBins + kBins / 32) * kTopkChunk * 4;   // [bin][column of the chunk]; the selection step re-uses it padded
+constexpr unsigned long long kKeyTop = 3ull << 62;              // the two always-set top bits of a key
 
 __device__ __forceinline__ unsigned long long make_key(float s, int64_t t) {
   return ((unsigned long long)(~__float_as_uint(s)) << 32) | (unsigned long long)(unsigned)t;
 }
 
 struct TopkLayout {
-  size_t off_state, off_hist, off_counters, off_cursor, off_keys, zero_bytes, total;
+  size_t off_state, off_hist, off_counters, off_cursor, off_cand, off_keys, zero_bytes, total;
   int chunks; int64_t kpad;
 };
 static TopkLayout topk_layout(int64_t n, int E, int64_t k) {
@@ -157,23 +164,65 @@ static TopkLayout topk_layout(int64_t n, int E, int64_t k) {
   size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += (b + 255) & ~(size_t)255; return r; };
   L.off_state = take(sizeof(SelState) * (size_t)E);
-  L.off_hist = take((size_t)kRadixPasses * E * 256 * 4);
+  L.off_hist = take((size_t)E * kBins * 4);
   L.off_counters = take((size_t)kRadixPasses * L.chunks * 4);
-  L.off_cursor = take((size_t)E * 4);
+  L.off_cursor = take((size_t)2 * E * 4);
   L.zero_bytes = o;                       // everything up to here starts at zero
+  L.off_cand = take((size_t)E * kCandCap * 8);
   L.off_keys = take((size_t)E * L.kpad * 8);
   L.total = o;
   return L;
 }
 size_t topk_scratch_bytes(int64_t n, int E, int64_t k) { return topk_layout(n, E, k).total; }
 
-// maps the lanes of a warp on a [rows x cw] slab of S: cwp = power of two >= cw
 __device__ __forceinline__ int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
-__global__ void __launch_bounds__(kHistThreads)
+// Walks the [t0, t1) x [c0, c0 + cw) slab of S with every thread of the CTA and calls f(score, token,
+// column within the chunk).  VEC: 16-byte loads (E a multiple of 4), else scalar.  Four independent
+// loads per thread are in flight.
+template <bool VEC, typename F>
+__device__ __forceinline__ void for_slab(const float* __restrict__ S, int E, int c0, int cw, int64_t t0, int64_t t1, F&& f) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  constexpr int U = 4;
+  if constexpr (VEC) {
+    const int lpr = pow2_at_least((cw + 3) >> 2), rpw = 32 / lpr;      // lanes per row, rows per warp
+    const int r = lane / lpr, g = (lane % lpr) * 4;
+    if (g >= cw) return;
+    const int64_t step = (int64_t)nwarps * rpw;
+    for (int64_t t = t0 + warp * rpw + r; t < t1; t += step * U) {
+      float4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (t + u * step < t1) v[u] = *reinterpret_cast<const float4*>(S + (t + u * step) * E + c0 + g);
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (t + u * step < t1) {
+          const int64_t tt = t + u * step;
+          f(v[u].x, tt, g); f(v[u].y, tt, g + 1); f(v[u].z, tt, g + 2); f(v[u].w, tt, g + 3);
+        }
+    }
+  } else {
+    const int cwp = pow2_at_least(cw), rpw = 32 / cwp;
+    const int r = lane / cwp, cc = lane % cwp;
+    if (cc >= cw) return;
+    const int64_t step = (int64_t)nwarps * rpw;
+    for (int64_t t = t0 + warp * rpw + r; t < t1; t += step * U) {
+      float v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (t + u * step < t1) v[u] = S[(t + u * step) * E + c0 + cc];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (t + u * step < t1) f(v[u], t + u * step, cc);
+    }
+  }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kHistThreads, 1)
 topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int pass, int rows_per_cta,
                  SelState* state, unsigned* hist, unsigned* counters) {
-  __shared__ unsigned sh[256 * kTopkChunk];            // [digit][column]
+  extern __shared__ unsigned sh[];                     // [bin][column]
   __shared__ unsigned long long s_prefix[kTopkChunk];
   __shared__ int s_active[kTopkChunk];
   __shared__ int s_any, s_last;
@@ -185,33 +234,27 @@ topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int 
     int act = 0; unsigned long long pre = 0;
     if (tid < cw) {
       if (pass == 0) act = 1;
-      else { act = state[c0 + tid].done ? 0 : 1; pre = state[c0 + tid].prefix; }
+      else { act = state[c0 + tid].mode == 0 ? 1 : 0; pre = state[c0 + tid].prefix; }
     }
     s_active[tid] = act; s_prefix[tid] = pre;
     if (act) s_any = 1;
   }
-  for (int i = tid; i < 256 * kTopkChunk; i += kHistThreads) sh[i] = 0;
+  for (int i = tid; i < kBins * kTopkChunk; i += kHistThreads) sh[i] = 0;
   __syncthreads();
-  if (!s_any) return;                                  // uniform: every expert of the chunk is finished
-  const int shift = 56 - 8 * pass;
-  const int cwp = pow2_at_least(cw), rpw = 32 / cwp;
-  const int warp = tid >> 5, lane = tid & 31, nwarps = kHistThreads / 32;
-  const int r = lane / cwp, cc = lane % cwp;
+  if (!s_any) return;                                  // uniform: every expert of the chunk is decided
+  const int shift = 52 - kRadixBits * pass;            // score bits 29..20, 19..10, 9..0
   const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
   const int64_t t1 = min(n, t0 + rows_per_cta);
-  if (cc < cw && s_active[cc]) {
-    const unsigned long long pre = s_prefix[cc];
-    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw) {
-      const unsigned long long key = make_key(S[t * E + c0 + cc], t);
-      const bool match = pass == 0 || ((key ^ pre) >> (shift + 8)) == 0;
-      if (match) atomicAdd(&sh[(unsigned)((key >> shift) & 255) * kTopkChunk + cc], 1u);
-    }
-  }
+  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
+    if (!s_active[col]) return;
+    const unsigned long long key = make_key(s, t);
+    const bool match = pass == 0 || ((key ^ s_prefix[col]) >> (shift + kRadixBits)) == 0;
+    if (match) atomicAdd(&sh[(unsigned)((key >> shift) & (kBins - 1)) * kTopkChunk + col], 1u);
+  });
   __syncthreads();
-  for (int i = tid; i < 256 * kTopkChunk; i += kHistThreads) {
+  for (int i = tid; i < kBins * kTopkChunk; i += kHistThreads) {
     const unsigned v = sh[i];
-    const int col = i % kTopkChunk, dig = i / kTopkChunk;
-    if (v) atomicAdd(&hist[((size_t)pass * E + c0 + col) * 256 + dig], v);
+    if (v) atomicAdd(&hist[(size_t)(c0 + i % kTopkChunk) * kBins + i / kTopkChunk], v);
   }
   __threadfence();
   __syncthreads();
@@ -219,75 +262,133 @@ topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int 
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // The last CTA of this chunk sees the full histograms: descend one digit per active expert.
-  for (int col = warp; col < cw; col += nwarps) {
-    if (!s_active[col]) continue;
-    const unsigned* h = hist + ((size_t)pass * E + c0 + col) * 256;
-    unsigned cnt[8], lsum = 0;
+  // The last CTA of this chunk sees the full histograms: one warp per expert finds the bucket of the
+  // k-th key, records the decision and leaves the histogram zeroed for the next pass.
+  const int warp = tid >> 5, lane = tid & 31;
+  if (warp >= cw || !s_active[warp]) return;
+  // The expert's kBins counts come in with coalesced, independent loads (lane holds bins lane, 32 + lane, ...),
+  // are laid out in the CTA's shared histogram (free by now; one padding word per 32 keeps the banks
+  // apart) and are read back as 32 consecutive bins per lane.
+  unsigned* h = hist + (size_t)(c0 + warp) * kBins;
+  constexpr int PER = kBins / 32;
+  unsigned* col = sh + warp * (kBins + PER);
+  {
+    unsigned tmp[PER];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { cnt[j] = __ldcg(h + lane * 8 + j); lsum += cnt[j]; }
-    unsigned incl = lsum;
-    for (int o = 1; o < 32; o <<= 1) { const unsigned v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-    const unsigned excl = incl - lsum;
-    const unsigned k_rem = pass == 0 ? k : state[c0 + col].k_rem;
-    if (excl < k_rem && k_rem <= incl) {               // exactly one lane
-      unsigned before = excl; int D = 0;
+    for (int j = 0; j < PER; ++j) tmp[j] = __ldcg(h + j * 32 + lane);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        if (before < k_rem && k_rem <= before + cnt[j]) { D = j; break; }
-        before += cnt[j];
-      }
-      const unsigned in_bucket = cnt[D];
-      const unsigned new_rem = k_rem - before;
-      unsigned long long pre = s_prefix[col] | ((unsigned long long)(lane * 8 + D) << shift);
-      SelState ns;
-      ns.k_rem = new_rem;
-      ns.done = (in_bucket == new_rem) ? 1u : 0u;
-      if (ns.done && shift > 0) pre |= (1ull << shift) - 1ull;   // whole bucket is taken
-      ns.prefix = pre;
-      state[c0 + col] = ns;
+    for (int j = 0; j < PER; ++j) { h[j * 32 + lane] = 0; col[j * 33 + lane] = tmp[j]; }
+  }
+  __syncwarp();
+  unsigned lsum = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) lsum += col[lane * 33 + j];
+  unsigned incl = lsum;
+  for (int o = 1; o < 32; o <<= 1) { const unsigned v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+  const unsigned excl = incl - lsum;
+  const unsigned k_rem = pass == 0 ? k : state[c0 + warp].k_rem;
+  if (excl < k_rem && k_rem <= incl) {                 // exactly one lane
+    unsigned before = excl, in_bucket = 0; int D = 0;
+    for (int j = 0; j < PER; ++j) {
+      const unsigned c = col[lane * 33 + j];
+      if (k_rem <= before + c) { D = j; in_bucket = c; break; }
+      before += c;
     }
+    const unsigned new_rem = k_rem - before;
+    SelState ns;
+    ns.prefix = (pass == 0 ? kKeyTop : s_prefix[warp]) | ((unsigned long long)(lane * PER + D) << shift);
+    ns.shift = (unsigned)shift; ns.k_rem = new_rem; ns.cand = 0;
+    if (in_bucket == new_rem) ns.mode = 1;                             // the whole bucket is taken
+    else if (in_bucket <= (unsigned)kCandCap) { ns.mode = 2; ns.cand = in_bucket; }   // the sort picks new_rem of these
+    else ns.mode = 0;                                                  // descend one more digit
+    state[c0 + warp] = ns;
   }
 }
 
-// Copies the keys not above each expert's threshold to keys[i][0..k), in no particular order.
+// Experts undecided after the score passes: more than kCandCap keys share the threshold score exactly,
+// and the k_rem lowest tokens among them win.  One CTA per expert walks the column in token order.
+__global__ void __launch_bounds__(1024)
+topk_ties_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int64_t kpad, SelState* state,
+                 unsigned long long* keys) {
+  __shared__ unsigned s_warp[32];
+  __shared__ unsigned s_total;
+  const int e = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (state[e].mode != 0) return;
+  const unsigned thr = (unsigned)(state[e].prefix >> 32), k_rem = state[e].k_rem, k_def = k - k_rem;
+  unsigned running = 0;
+  for (int64_t base = 0; base < n && running < k_rem; base += 1024) {
+    const int64_t t = base + tid;
+    float s = 0.f; bool m = false;
+    if (t < n) { s = S[t * E + e]; m = ~__float_as_uint(s) == thr; }
+    const unsigned bal = __ballot_sync(0xffffffffu, m);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      const unsigned v = s_warp[lane];
+      unsigned inc = v;
+      for (int o = 1; o < 32; o <<= 1) { const unsigned u = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += u; }
+      s_warp[lane] = inc - v;
+      if (lane == 31) s_total = inc;
+    }
+    __syncthreads();
+    const unsigned idx = running + s_warp[warp] + __popc(bal & ((1u << lane) - 1u));
+    if (m && idx < k_rem) keys[(size_t)e * kpad + k_def + idx] = make_key(s, t);
+    running += s_total;
+    __syncthreads();
+  }
+  if (tid == 0) state[e].mode = 3;
+}
+
+// Copies each expert's winners to keys[i][0 ..) and its candidates to cand[i][0 ..), in no particular order.
+template <bool VEC>
 __global__ void __launch_bounds__(kHistThreads)
-topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int64_t kpad,
-                    int rows_per_cta, const SelState* __restrict__ state, unsigned* cursor,
-                    unsigned long long* keys) {
-  __shared__ unsigned s_cnt[kTopkChunk], s_base[kTopkChunk];
+topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int64_t kpad, int rows_per_cta,
+                    const SelState* __restrict__ state, unsigned* cursor, unsigned long long* keys,
+                    unsigned long long* cand) {
+  __shared__ unsigned s_cnt[2][kTopkChunk], s_base[2][kTopkChunk];
   __shared__ unsigned long long s_thr[kTopkChunk];
+  __shared__ unsigned s_shift[kTopkChunk], s_mode[kTopkChunk];
   const int tid = threadIdx.x, chunk = blockIdx.y;
   const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
-  if (tid < kTopkChunk) { s_cnt[tid] = 0; s_thr[tid] = tid < cw ? state[c0 + tid].prefix : 0ull; }
-  __syncthreads();
-  const int cwp = pow2_at_least(cw), rpw = 32 / cwp;
-  const int warp = tid >> 5, lane = tid & 31, nwarps = kHistThreads / 32;
-  const int r = lane / cwp, cc = lane % cwp;
-  const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
-  const int64_t t1 = min(n, t0 + rows_per_cta);
-  unsigned long long thr = 0;
-  if (cc < cw) {
-    thr = s_thr[cc];
-    unsigned mine = 0;
-    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw)
-      mine += make_key(S[t * E + c0 + cc], t) <= thr ? 1u : 0u;
-    if (mine) atomicAdd(&s_cnt[cc], mine);
-  }
-  __syncthreads();
-  if (tid < cw) { const unsigned c = s_cnt[tid]; s_base[tid] = c ? atomicAdd(&cursor[c0 + tid], c) : 0u; }
-  __syncthreads();
-  if (tid < kTopkChunk) s_cnt[tid] = 0;
-  __syncthreads();
-  if (cc < cw) {
-    for (int64_t t = t0 + warp * rpw + r; t < t1; t += nwarps * rpw) {
-      const unsigned long long key = make_key(S[t * E + c0 + cc], t);
-      if (key <= thr) {
-        const unsigned pos = s_base[cc] + atomicAdd(&s_cnt[cc], 1u);
-        if (pos < k) keys[(size_t)(c0 + cc) * kpad + pos] = key;
-      }
+  if (tid < kTopkChunk) {
+    s_cnt[0][tid] = s_cnt[1][tid] = 0;
+    if (tid < cw) {
+      const SelState st = state[c0 + tid];
+      s_shift[tid] = st.shift; s_thr[tid] = st.prefix >> st.shift; s_mode[tid] = st.mode;
     }
   }
+  __syncthreads();
+  const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
+  const int64_t t1 = min(n, t0 + rows_per_cta);
+  // 0: not taken, 1: winner, 2: candidate
+  auto classify = [&](float s, int64_t t, int col) -> int {
+    const unsigned long long hi = make_key(s, t) >> s_shift[col];
+    if (hi < s_thr[col]) return 1;
+    if (hi > s_thr[col]) return 0;
+    return s_mode[col] == 1 ? 1 : (s_mode[col] == 2 ? 2 : 0);          // mode 3: the tie walk placed them
+  };
+  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
+    const int c = classify(s, t, col);
+    if (c) atomicAdd(&s_cnt[c - 1][col], 1u);
+  });
+  __syncthreads();
+  if (tid < 2 * kTopkChunk) {
+    const int w = tid / kTopkChunk, col = tid % kTopkChunk;
+    if (col < cw) { const unsigned c = s_cnt[w][col]; s_base[w][col] = c ? atomicAdd(&cursor[w * E + c0 + col], c) : 0u; }
+  }
+  __syncthreads();
+  if (tid < kTopkChunk) s_cnt[0][tid] = s_cnt[1][tid] = 0;
+  __syncthreads();
+  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
+    const int c = classify(s, t, col);
+    if (c == 1) {
+      const unsigned pos = s_base[0][col] + atomicAdd(&s_cnt[0][col], 1u);
+      if (pos < k) keys[(size_t)(c0 + col) * kpad + pos] = make_key(s, t);
+    } else if (c == 2) {
+      const unsigned pos = s_base[1][col] + atomicAdd(&s_cnt[1][col], 1u);
+      if (pos < (unsigned)kCandCap) cand[(size_t)(c0 + col) * kCandCap + pos] = make_key(s, t);
+    }
+  });
 }
 
 __device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, float* G, int64_t o) {
@@ -295,9 +396,66 @@ __device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, fl
   G[o] = __uint_as_float(~(unsigned)(key >> 32));
 }
 
+// Ascending bitonic sort of len (a power of two) keys in shared memory by the whole CTA.
+__device__ __forceinline__ void bitonic_smem(unsigned long long* a, int len) {
+  for (int size = 2; size <= len; size <<= 1) {
+    for (int stride = size >> 1; stride >= 1; stride >>= 1) {
+      for (int p = threadIdx.x; p < (len >> 1); p += blockDim.x) {
+        const int i = (p / stride) * 2 * stride + (p % stride), j = i + stride;
+        const bool asc = (i & size) == 0;
+        const unsigned long long x = a[i], y = a[j];
+        if ((x > y) == asc) { a[i] = y; a[j] = x; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Sorts an expert's candidates and returns (in shared memory) them in ascending order; sc holds kCandCap keys.
+__device__ __forceinline__ void load_sorted_candidates(const unsigned long long* cand, int e, unsigned ncand,
+                                                       unsigned long long* sc) {
+  const int len = pow2_at_least((int)ncand);
+  for (int i = threadIdx.x; i < len; i += blockDim.x) sc[i] = i < (int)ncand ? cand[(size_t)e * kCandCap + i] : ~0ull;
+  __syncthreads();
+  bitonic_smem(sc, len);
+}
+
+// k up to one tile: one CTA per expert merges the candidates in, sorts the k keys and writes I and G.
+constexpr int kSortThreads = 1024;
+__global__ void __launch_bounds__(kSortThreads)
+topk_finish_tile_kernel(const unsigned long long* __restrict__ keys, const unsigned long long* __restrict__ cand,
+                        const SelState* __restrict__ state, int64_t kpad, int64_t k, int32_t* I, float* G) {
+  __shared__ unsigned long long sk[kSortTile];
+  __shared__ unsigned long long sc[kCandCap];
+  const int e = blockIdx.x;
+  const SelState st = state[e];
+  for (int i = threadIdx.x; i < kpad; i += kSortThreads) sk[i] = keys[(size_t)e * kpad + i];
+  __syncthreads();
+  if (st.mode == 2) {
+    load_sorted_candidates(cand, e, st.cand, sc);
+    const unsigned k_def = (unsigned)k - st.k_rem;
+    for (int i = threadIdx.x; i < (int)st.k_rem; i += kSortThreads) sk[k_def + i] = sc[i];
+    __syncthreads();
+  }
+  bitonic_smem(sk, (int)kpad);
+  for (int i = threadIdx.x; i < k; i += kSortThreads) emit_slot(sk[i], I, G, (int64_t)e * k + i);
+}
+
+// k beyond one tile: the candidates are merged into the global key list first.
+__global__ void __launch_bounds__(kSortThreads)
+topk_resolve_kernel(unsigned long long* keys, const unsigned long long* __restrict__ cand,
+                    const SelState* __restrict__ state, int64_t kpad, int64_t k) {
+  __shared__ unsigned long long sc[kCandCap];
+  const int e = blockIdx.x;
+  const SelState st = state[e];
+  if (st.mode != 2) return;
+  load_sorted_candidates(cand, e, st.cand, sc);
+  const unsigned k_def = (unsigned)k - st.k_rem;
+  for (int i = threadIdx.x; i < (int)st.k_rem; i += kSortThreads) keys[(size_t)e * kpad + k_def + i] = sc[i];
+}
+
 // Bitonic steps on one tile of kSortTile keys held in shared memory.  Runs the network sizes
 // size_lo..size_hi (powers of two); for a size larger than the tile only the strides that fit.
-constexpr int kSortThreads = 1024;
 __global__ void __launch_bounds__(kSortThreads)
 topk_sort_tile_kernel(unsigned long long* keys, int64_t kpad, int64_t k, int64_t size_lo, int64_t size_hi,
                       int emit, int32_t* I, float* G) {
@@ -351,26 +509,37 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I,
   unsigned* hist = (unsigned*)(base + L.off_hist);
   unsigned* counters = (unsigned*)(base + L.off_counters);
   unsigned* cursor = (unsigned*)(base + L.off_cursor);
+  unsigned long long* cand = (unsigned long long*)(base + L.off_cand);
   unsigned long long* keys = (unsigned long long*)(base + L.off_keys);
   cudaError_t e;
+  const bool vec = E % 4 == 0 && ((uintptr_t)S & 15) == 0;
+  // the histogram kernels use 128 KiB of dynamic shared memory
+  if ((e = vec ? cudaFuncSetAttribute(topk_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSmemBytes)
+               : cudaFuncSetAttribute(topk_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSmemBytes)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(base, 0, L.zero_bytes, st)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(keys, 0xFF, (size_t)E * L.kpad * 8, st)) != cudaSuccess) return e;
-  // rows per CTA: enough CTAs to fill the machine a few times over, at least 64 rows each
-  int64_t want = (int64_t)148 * 8 / L.chunks; if (want < 1) want = 1;
-  int64_t rows = (n + want - 1) / want; if (rows < 64) rows = 64;
+  // rows per CTA: about two CTAs per SM over all chunks, at least 256 rows each
+  int64_t want = (int64_t)148 * 2 / L.chunks; if (want < 1) want = 1;
+  int64_t rows = (n + want - 1) / want; if (rows < 256) rows = 256;
   const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks);
   for (int pass = 0; pass < kRadixPasses; ++pass) {
     count_launch();
-    topk_hist_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
+    if (vec) topk_hist_kernel<true><<<grid, kHistThreads, kHistSmemBytes, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
+    else topk_hist_kernel<false><<<grid, kHistThreads, kHistSmemBytes, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
   }
   count_launch();
-  topk_compact_kernel<<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys);
-  const int64_t tiles = (L.kpad + kSortTile - 1) / kSortTile;
-  const unsigned sort_grid = (unsigned)(E * tiles);
+  topk_ties_kernel<<<E, 1024, 0, st>>>(S, n, E, (unsigned)k, L.kpad, state, keys);
+  count_launch();
+  if (vec) topk_compact_kernel<true><<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys, cand);
+  else topk_compact_kernel<false><<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys, cand);
   if (L.kpad <= kSortTile) {
     count_launch();
-    topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, L.kpad, 1, I, G);
+    topk_finish_tile_kernel<<<E, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k, I, G);
   } else {
+    const int64_t tiles = (L.kpad + kSortTile - 1) / kSortTile;
+    const unsigned sort_grid = (unsigned)(E * tiles);
+    count_launch();
+    topk_resolve_kernel<<<E, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k);
     count_launch();
     topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, kSortTile, 0, I, G);
     const int64_t pairs = (int64_t)E * (L.kpad >> 1);
@@ -390,41 +559,74 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I,
 // Index form of P = Onehot(I) (Eq. 2) read by token: row_ptr / slots.
 // Integer atomics only count and hand out positions; each token's short list is then sorted,
 // so the result does not depend on the order in which threads ran.
-// scratch: [cursor n int32]
+// scratch: [cnt n+1 int32][tile sums ceil(n / kScanTile) int32]
 // ------------------------------------------------------------------------------------------
-size_t inverse_scratch_bytes(int64_t n) { return ((size_t)(n + 1) * 4 + 255) & ~(size_t)255; }
+constexpr int kScanTile = 4096, kScanThreads = 1024;
+static size_t inv_cnt_bytes(int64_t n) { return ((size_t)(n + 1) * 4 + 255) & ~(size_t)255; }
+size_t inverse_scratch_bytes(int64_t n) {
+  return inv_cnt_bytes(n) + ((((size_t)(n + kScanTile - 1) / kScanTile) * 4 + 255) & ~(size_t)255);
+}
 
 __global__ void inv_count_kernel(const int32_t* __restrict__ I, int64_t total, int32_t* cnt) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x)
     atomicAdd(&cnt[I[s]], 1);
 }
 
-// exclusive scan of cnt[0..n) into row_ptr[0..n], single CTA
-__global__ void __launch_bounds__(1024) inv_scan_kernel(const int32_t* __restrict__ cnt, int64_t n, int32_t* row_ptr) {
-  __shared__ int s_sum[1024];
-  const int tid = threadIdx.x;
-  const int64_t per = (n + 1023) / 1024;
-  const int64_t a = min(n, tid * per), b = min(n, a + per);
-  int sum = 0;
-  for (int64_t t = a; t < b; ++t) sum += cnt[t];
-  s_sum[tid] = sum;
+// Exclusive scan of the CTA's per-thread values (any thread count that is a multiple of 32, at most 1024);
+// returns the thread's offset and, in `total`, the sum over the CTA.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  int inc = v;
+  for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += u; }
+  if (lane == 31) s_warp[warp] = inc;
   __syncthreads();
-  for (int o = 1; o < 1024; o <<= 1) {
-    const int v = tid >= o ? s_sum[tid - o] : 0;
-    __syncthreads();
-    s_sum[tid] += v;
-    __syncthreads();
+  if (warp == 0) {
+    const int w = lane < nwarps ? s_warp[lane] : 0;
+    int winc = w;
+    for (int o = 1; o < 32; o <<= 1) { const int u = __shfl_up_sync(0xffffffffu, winc, o); if (lane >= o) winc += u; }
+    s_warp[lane] = winc - w;
+    if (lane == 31) s_warp[32] = winc;
   }
-  int run = s_sum[tid] - sum;
-  for (int64_t t = a; t < b; ++t) { row_ptr[t] = run; run += cnt[t]; }
-  if (tid == 1023) row_ptr[n] = s_sum[1023];
+  __syncthreads();
+  total = s_warp[32];
+  return s_warp[warp] + inc - v;
 }
 
+// Step 1: exclusive scan inside each tile of kScanTile counts (four per thread), tile sums aside.
+__global__ void __launch_bounds__(kScanThreads) inv_scan_tile_kernel(const int32_t* __restrict__ cnt, int64_t n,
+                                                                      int32_t* row_ptr, int32_t* tile_sum) {
+  __shared__ int s_warp[33];
+  const int64_t base = (int64_t)blockIdx.x * kScanTile + threadIdx.x * 4;
+  int c[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) c[j] = base + j < n ? cnt[base + j] : 0;
+  int total;
+  int run = block_exclusive_scan(c[0] + c[1] + c[2] + c[3], s_warp, total);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { if (base + j < n) row_ptr[base + j] = run; run += c[j]; }
+  if (threadIdx.x == 0) tile_sum[blockIdx.x] = total;
+}
+
+// Step 2: every tile adds the sum of the tiles before it; the last one also writes row_ptr[n].
+__global__ void __launch_bounds__(kScanThreads) inv_scan_add_kernel(const int32_t* __restrict__ tile_sum, int64_t n,
+                                                                     int32_t* row_ptr) {
+  __shared__ int s_warp[33];
+  int part = 0;
+  for (int j = threadIdx.x; j < (int)blockIdx.x; j += kScanThreads) part += tile_sum[j];
+  int before;
+  block_exclusive_scan(part, s_warp, before);
+  const int64_t base = (int64_t)blockIdx.x * kScanTile + threadIdx.x * 4;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) if (base + j < n) row_ptr[base + j] += before;
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) row_ptr[n] = before + tile_sum[blockIdx.x];
+}
+
+// Hands each slot a place in its token's list, counting the token's counter back down to zero.
 __global__ void inv_fill_kernel(const int32_t* __restrict__ I, int64_t total, const int32_t* __restrict__ row_ptr,
-                                int32_t* cursor, int32_t* slots) {
+                                int32_t* cnt, int32_t* slots) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
     const int t = I[s];
-    slots[row_ptr[t] + atomicAdd(&cursor[t], 1)] = (int32_t)s;
+    slots[row_ptr[t] + atomicSub(&cnt[t], 1) - 1] = (int32_t)s;
   }
 }
 
@@ -441,17 +643,19 @@ __global__ void inv_sort_kernel(const int32_t* __restrict__ row_ptr, int64_t n, 
 
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int32_t* row_ptr, int32_t* slots,
                                  void* scratch, cudaStream_t st) {
-  int32_t* cursor = (int32_t*)scratch;
+  int32_t* cnt = (int32_t*)scratch;
+  int32_t* tile_sum = (int32_t*)((char*)scratch + inv_cnt_bytes(n));
+  const unsigned tiles = (unsigned)((n + kScanTile - 1) / kScanTile);
   cudaError_t e;
-  // counts are built in slots' neighbour: reuse row_ptr[1..n] would break the scan, so count in `cursor`
-  if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(cnt, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
   count_launch();
-  inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cursor);
+  inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cnt);
   count_launch();
-  inv_scan_kernel<<<1, 1024, 0, st>>>(cursor, n, row_ptr);
-  if ((e = cudaMemsetAsync(cursor, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
+  inv_scan_tile_kernel<<<tiles, kScanThreads, 0, st>>>(cnt, n, row_ptr, tile_sum);
   count_launch();
-  inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cursor, slots);
+  inv_scan_add_kernel<<<tiles, kScanThreads, 0, st>>>(tile_sum, n, row_ptr);
+  count_launch();
+  inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cnt, slots);
   count_launch();
   inv_sort_kernel<<<grid_for(n, 256), 256, 0, st>>>(row_ptr, n, slots);
   return cudaGetLastError();

@@ -1,0 +1,64 @@
+"""The two remaining workload families, through the C ABI on a B200:
+
+  - routing-only stress (gate + softmax, column top-k, inverse index, shuffle, unshuffle with
+    identity experts, X_e = X_in) at d = 1024, bf16, over a grid of group sizes and expert counts;
+  - the capacity-factor sweep of the forward pass (E = 64, c in {0.5, 1, 2}, gate logits scaled
+    x1 and x4 to vary the skew of the scores).
+
+Routing and the index lists are compared bit for bit with the oracle evaluated on the GPU's own
+S; the shuffle is a copy and must be exact; the unshuffle is compared with the fp64 sum of
+Eq. 4 within the final bf16 rounding.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ec_oracle as O
+from paper_2202_09368_b200 import binding as B
+from paper_2202_09368_b200 import inputs as IN
+
+from _parity import TOL, check_routing, rel_err, run_and_check, to_np
+
+pytestmark = pytest.mark.gpu
+BF16 = torch.bfloat16
+
+
+@pytest.mark.parametrize("n,E", [(4096, 8), (4096, 32), (4096, 128), (4096, 256), (16384, 32), (16384, 256),
+                                 (65536, 8), (65536, 128)])
+def test_routing_only_chain_identity_experts(n, E):
+    d, c = 1024, 2.0
+    li = IN.make_layer_inputs(n, d, 8, E, BF16, seed=0, with_grad=False)
+    cfg = B.make_config(n, d, 8, E, c, BF16)
+    k = B.ec_capacity(cfg)
+    X, Wg = li.X.cuda(), li.Wg.cuda()
+    r = B.ec_route(cfg, X, Wg)
+    Xn, Wgn = to_np(li.X), to_np(li.Wg)
+    assert rel_err(to_np(r.S), O.gate(Xn, Wgn)) <= TOL[BF16]
+    I = check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+    # perfect load balance: k distinct tokens per expert, n*c slots in all
+    assert all(len(set(row)) == k for row in I[:: max(1, E // 8)])
+    assert int(r.row_ptr[-1]) == E * k == int(n * c)
+    # Eq. 3 with P as an index list: a copy
+    X_in = B.ec_shuffle(cfg, X, r.I)
+    assert torch.equal(X_in, X[r.I.long()])
+    # Eq. 4 with identity experts
+    X_e = X_in.float()
+    X_out = B.ec_unshuffle(cfg, X_e, r.G, r.row_ptr, r.slots)
+    G = to_np(r.G).reshape(-1)
+    ref = np.zeros((n, d))
+    np.add.at(ref, I.reshape(-1), G[:, None] * Xn[I.reshape(-1)])          # fp64 sum over the slots of each token
+    got = to_np(X_out)
+    scale = np.sqrt(np.mean(ref ** 2))
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-6 * scale)      # one bf16 rounding
+    cnt = to_np(r.row_ptr)[1:] - to_np(r.row_ptr)[:-1]
+    assert torch.all(X_out[torch.from_numpy(cnt == 0).cuda()] == 0)
+
+
+@pytest.mark.parametrize("c", [0.5, 1.0, 2.0])
+@pytest.mark.parametrize("scale", [1.0, 4.0])
+def test_capacity_factor_sweep_forward(c, scale):
+    n, d, dff, E = 8192, 768, 3072, 64
+    li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=0, logit_scale=scale, with_grad=False, device="cuda")
+    errs = run_and_check(n, d, dff, E, c, BF16, li, backward=False)
+    assert B.ec_capacity(B.make_config(n, d, dff, E, c, BF16)) == int(n * c / E)
+    print(c, scale, {k_: (f"{v:.3e}" if not isinstance(v, dict) else v) for k_, v in errs.items()})
