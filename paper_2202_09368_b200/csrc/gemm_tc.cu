@@ -231,13 +231,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmC2, const TcParams p) {
   constexpr int BNL = BN / CTAS;                    // rows of B this CTA loads
   constexpr int TM = BM * CTAS;                     // rows of the tile the CTA (pair) works on
-  constexpr int S = num_stages(BNL);
+  constexpr bool kXchg = EPI == EPI_SOFTMAX && BN >= 128;            // the softmax epilogue's exchange area replaces a stage
+  constexpr int S = num_stages(BNL) - (kXchg ? 1 : 0);
   constexpr int kBBytes = BNL * BK * 2;
   constexpr int kStage = kABytes + kBBytes;
   constexpr int kCols = tmem_cols(BN, CTAS);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = (uint64_t*)(smem + S * kStage + kEpiWarps * kStagingPerWarp);   // full[S], empty[S], tmem_full[2], tmem_empty[2]
+  // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]; 256 bytes further on, with kXchg: [2][8 warps][32] float2, int[8]
+  uint64_t* bars = (uint64_t*)(smem + S * kStage + kEpiWarps * kStagingPerWarp);
   uint32_t* tmem_slot = (uint32_t*)(bars + 2 * S + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, tfull0 = empty0 + 8 * S, tempty0 = tfull0 + 16;
@@ -250,6 +252,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int s = 0; s < S; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, CTAS * kEpiWarps); }
     *abort_flag = 0;
+    if constexpr (kXchg) {
+      int* published = (int*)(smem + S * kStage + kEpiWarps * kStagingPerWarp + 256 + 2 * kEpiWarps * 32 * 8);
+      for (int w = 0; w < kEpiWarps; ++w) published[w] = 0;
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -379,36 +385,83 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int n0 = nt * BN;
       const int64_t obase = (int64_t)b * p.batch_c + (int64_t)row * p.ldc;
       if constexpr (EPI == EPI_SOFTMAX) {
-       if (half == 0) {                             // a row's softmax stays in one thread
-        // Eq. 2: softmax over the N = E columns of this row; columns >= N are padding.
-        float mx = -INFINITY;
-        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
-          uint32_t r[32]; tc_ld32(taddr + c0, r);
+        // Eq. 2: softmax over the N = E columns of each row; columns >= N are padding.  A thread owns one
+        // row.  With BN >= 128 the two warps of a lane quarter take half of the columns each and exchange
+        // their (max, sum) through shared memory.  First sweep over tensor memory: running max and sum
+        // of exp(x - max); second sweep: exp(x - max) / sum, staged and stored like any fp32 result.
+        constexpr bool kSplit = BN >= 128;
+        constexpr int kColsPerWarp = kSplit ? BN / 2 : BN;
+        const int cbeg = kSplit ? half * kColsPerWarp : 0;
+        const bool active = kSplit || half == 0;
+        uint8_t* stg = smem + S * kStage + (warp - 2) * kStagingPerWarp;
+        const uint32_t stg_s = smem_u32(stg);
+        const int r0 = mt * TM + (int)rank * BM + q * 32;
+        float mx = -INFINITY, sum = 0.f;
+        if (active) {
+#pragma unroll 1
+          for (int c0 = cbeg; c0 < cbeg + kColsPerWarp && c0 < p.N; c0 += 32) {
+            uint32_t r[32]; tc_ld32(taddr + c0, r);
+            float cm = -INFINITY;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (c0 + j < p.N) mx = fmaxf(mx, __uint_as_float(r[j]));
-        }
-        float sum = 0.f;
-        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
-          uint32_t r[32]; tc_ld32(taddr + c0, r);
+            for (int j = 0; j < 32; ++j) if (c0 + j < p.N) cm = fmaxf(cm, __uint_as_float(r[j]));
+            const float mn = fmaxf(mx, cm);
+            float part = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (c0 + j < p.N) sum += expf(__uint_as_float(r[j]) - mx);
-        }
-        const float inv = 1.f / sum;
-        for (int c0 = 0; c0 < BN && c0 < p.N; c0 += 32) {
-          uint32_t r[32]; tc_ld32(taddr + c0, r);
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              if (c0 + j < p.N) {          // N is a multiple of 8
-                float4 o;
-                o.x = expf(__uint_as_float(r[j]) - mx) * inv; o.y = expf(__uint_as_float(r[j + 1]) - mx) * inv;
-                o.z = expf(__uint_as_float(r[j + 2]) - mx) * inv; o.w = expf(__uint_as_float(r[j + 3]) - mx) * inv;
-                *reinterpret_cast<float4*>(p.S + (int64_t)row * p.ldc + c0 + j) = o;
-              }
-            }
+            for (int j = 0; j < 32; ++j) if (c0 + j < p.N) part += __expf(__uint_as_float(r[j]) - mn);
+            sum = sum * __expf(mx - mn) + part;
+            mx = mn;
           }
         }
-       }
+        if constexpr (kSplit) {
+          // The partner's (max, sum) comes through a slot in shared memory, one per warp and tile parity, with
+          // a per-warp counter of published tiles.  A slot is rewritten two tiles later, which the partner's
+          // release of the accumulator (it precedes that tile's MMAs) orders after its read.  The wait is bounded.
+          float2* xch = reinterpret_cast<float2*>(smem + S * kStage + kEpiWarps * kStagingPerWarp + 256);
+          volatile int* published = reinterpret_cast<volatile int*>(xch + 2 * kEpiWarps * 32);
+          const int me = warp - 2, partner = me ^ 4;
+          xch[((it & 1) * kEpiWarps + me) * 32 + lane] = make_float2(mx, sum);
+          __threadfence_block();
+          __syncwarp();
+          if (lane == 0) published[me] = it + 1;
+          bool seen = published[partner] >= it + 1;
+          if (!seen) {
+            const unsigned long long t0 = globaltimer();
+            for (uint32_t spin = 1; !seen; ++spin) {
+              seen = published[partner] >= it + 1;
+              if (!seen && (spin & 63u) == 0 && (*abort_flag || globaltimer() - t0 > kWaitNs)) break;
+            }
+          }
+          if (!__all_sync(0xffffffffu, seen)) {
+            if (lane == 0) { *abort_flag = 1; atomicExch(p.status + 1, 7); atomicExch(p.status, 5); }
+            gave_up = true; break;
+          }
+          __threadfence_block();
+          const float2 o = xch[((it & 1) * kEpiWarps + partner) * 32 + lane];
+          const float mn = fmaxf(mx, o.x);
+          sum = sum * __expf(mx - mn) + (o.y > 0.f ? o.y * __expf(o.x - mn) : 0.f);
+          mx = mn;
+        }
+        const float inv = 1.f / sum;
+        const int sw = lane & 7;
+        if (active) {
+#pragma unroll 1
+          for (int c0 = cbeg; c0 < cbeg + kColsPerWarp && c0 < p.N; c0 += 32, ++nchunk) {
+            uint32_t r[32]; tc_ld32(taddr + c0, r);
+            uint8_t* bufp = stg + (nchunk & 1) * 4096;
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float4 o;
+              o.x = __expf(__uint_as_float(r[4 * j]) - mx) * inv; o.y = __expf(__uint_as_float(r[4 * j + 1]) - mx) * inv;
+              o.z = __expf(__uint_as_float(r[4 * j + 2]) - mx) * inv; o.w = __expf(__uint_as_float(r[4 * j + 3]) - mx) * inv;
+              *reinterpret_cast<float4*>(bufp + lane * 128 + ((j ^ sw) << 4)) = o;
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + (nchunk & 1) * 4096, c0, r0, 0); bulk_commit(); }
+          }
+        }
       } else {
         // Results leave through shared memory and the TMA unit.  A warp owns 32 rows and kColsPerWarp columns
         // of the tile and works on chunks whose rows are 128 bytes long (64 bf16 or 32 fp32 columns): each
@@ -576,11 +629,12 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
 
 int pick_bn(const TcGemmArgs& g) { return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64); }
 // Two CTAs per tile when a tile of 256 rows is not mostly padding and the pair's B halves are whole 64-wide blocks.
-int pick_ctas(const TcGemmArgs& g, int bn) { return (g.epi != EPI_SOFTMAX && bn >= 128 && g.M > BM) ? 2 : 1; }
+int pick_ctas(const TcGemmArgs& g, int bn) { return (bn >= 128 && g.M > BM) ? 2 : 1; }
 
 template <int BN, int EPI, int CTAS>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                        const TcParams& p, cudaStream_t st) {
+  // the split softmax trades one operand stage for its exchange area (4 KiB + counters), see the kernel
   constexpr int smem = num_stages(BN / CTAS) * stage_bytes(BN / CTAS) + kEpiWarps * kStagingPerWarp + 1024 + 256;
   auto kern = gemm_tc_kernel<BN, EPI, CTAS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -615,7 +669,7 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
 template <int EPI>
 cudaError_t launch_bn(int bn, int ctas, const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                       const TcParams& p, cudaStream_t st) {
-  if constexpr (EPI != EPI_SOFTMAX) {
+  {
     if (ctas == 2) {
       if (bn == 256) return launch_one<256, EPI, 2>(ta, tb, tc, tc2, p, st);
       return launch_one<128, EPI, 2>(ta, tb, tc, tc2, p, st);
@@ -657,7 +711,9 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   if (!oka || !okb) return cudaErrorInvalidValue;
   // outputs leave through TMA stores of chunks of 32 rows x 128 bytes (64 bf16 or 32 fp32 columns)
   CUtensorMap tc = ta, tc2 = ta;
-  if (g.epi != EPI_SOFTMAX) {
+  if (g.epi == EPI_SOFTMAX) {
+    if (!make_map(&tc, g.S, g.N, g.M, 1, g.ldc, 0, 32, 32, true)) return cudaErrorInvalidValue;
+  } else {
     if (!make_map(&tc, g.C, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, 32, g.c_f32 != 0)) return cudaErrorInvalidValue;
     if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 64, 32)) return cudaErrorInvalidValue;
   }

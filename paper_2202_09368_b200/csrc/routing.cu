@@ -339,17 +339,24 @@ topk_ties_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int6
   if (tid == 0) state[e].mode = 3;
 }
 
-// Copies each expert's winners to keys[i][0 ..) and its candidates to cand[i][0 ..), in no particular order.
+// Copies each expert's winners to keys[i][0 ..) and its candidates to cand[i][0 ..), in no particular
+// order, with one read of S: a CTA parks what it finds in shared memory, reserves one range per
+// (expert, kind) with a single global atomic each and writes the keys out.  What does not fit in the
+// buffer (only with very uneven inputs) takes its place with a global atomic of its own.
+constexpr int kCompactCap = 4096;
 template <bool VEC>
 __global__ void __launch_bounds__(kHistThreads)
 topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int64_t kpad, int rows_per_cta,
                     const SelState* __restrict__ state, unsigned* cursor, unsigned long long* keys,
                     unsigned long long* cand) {
-  __shared__ unsigned s_cnt[2][kTopkChunk], s_base[2][kTopkChunk];
+  __shared__ unsigned long long s_key[kCompactCap];
+  __shared__ unsigned char s_tag[kCompactCap];         // column within the chunk, bit 7: candidate
+  __shared__ unsigned s_cnt[2][kTopkChunk], s_base[2][kTopkChunk], s_n;
   __shared__ unsigned long long s_thr[kTopkChunk];
   __shared__ unsigned s_shift[kTopkChunk], s_mode[kTopkChunk];
   const int tid = threadIdx.x, chunk = blockIdx.y;
   const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
+  if (tid == 0) s_n = 0;
   if (tid < kTopkChunk) {
     s_cnt[0][tid] = s_cnt[1][tid] = 0;
     if (tid < cw) {
@@ -360,17 +367,24 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
   __syncthreads();
   const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
   const int64_t t1 = min(n, t0 + rows_per_cta);
-  // 0: not taken, 1: winner, 2: candidate
-  auto classify = [&](float s, int64_t t, int col) -> int {
-    const unsigned long long hi = make_key(s, t) >> s_shift[col];
-    if (hi < s_thr[col]) return 1;
-    if (hi > s_thr[col]) return 0;
-    return s_mode[col] == 1 ? 1 : (s_mode[col] == 2 ? 2 : 0);          // mode 3: the tie walk placed them
+  auto put = [&](int kind, int col, unsigned pos, unsigned long long key) {      // kind 0: winner, 1: candidate
+    if (kind == 0) { if (pos < k) keys[(size_t)(c0 + col) * kpad + pos] = key; }
+    else if (pos < (unsigned)kCandCap) cand[(size_t)(c0 + col) * kCandCap + pos] = key;
   };
   for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
-    const int c = classify(s, t, col);
-    if (c) atomicAdd(&s_cnt[c - 1][col], 1u);
+    const unsigned long long key = make_key(s, t), hi = key >> s_shift[col];
+    int kind;                                          // mode 3: the tie walk has placed the keys at the threshold
+    if (hi < s_thr[col]) kind = 0;
+    else if (hi == s_thr[col] && s_mode[col] == 1) kind = 0;
+    else if (hi == s_thr[col] && s_mode[col] == 2) kind = 1;
+    else return;
+    const unsigned idx = atomicAdd(&s_n, 1u);
+    if (idx < (unsigned)kCompactCap) { s_key[idx] = key; s_tag[idx] = (unsigned char)(col | (kind << 7)); }
+    else put(kind, col, atomicAdd(&cursor[kind * E + c0 + col], 1u), key);
   });
+  __syncthreads();
+  const int held = (int)min(s_n, (unsigned)kCompactCap);
+  for (int i = tid; i < held; i += kHistThreads) atomicAdd(&s_cnt[s_tag[i] >> 7][s_tag[i] & 127], 1u);
   __syncthreads();
   if (tid < 2 * kTopkChunk) {
     const int w = tid / kTopkChunk, col = tid % kTopkChunk;
@@ -379,16 +393,10 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
   __syncthreads();
   if (tid < kTopkChunk) s_cnt[0][tid] = s_cnt[1][tid] = 0;
   __syncthreads();
-  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
-    const int c = classify(s, t, col);
-    if (c == 1) {
-      const unsigned pos = s_base[0][col] + atomicAdd(&s_cnt[0][col], 1u);
-      if (pos < k) keys[(size_t)(c0 + col) * kpad + pos] = make_key(s, t);
-    } else if (c == 2) {
-      const unsigned pos = s_base[1][col] + atomicAdd(&s_cnt[1][col], 1u);
-      if (pos < (unsigned)kCandCap) cand[(size_t)(c0 + col) * kCandCap + pos] = make_key(s, t);
-    }
-  });
+  for (int i = tid; i < held; i += kHistThreads) {
+    const int kind = s_tag[i] >> 7, col = s_tag[i] & 127;
+    put(kind, col, s_base[kind][col] + atomicAdd(&s_cnt[kind][col], 1u), s_key[i]);
+  }
 }
 
 __device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, float* G, int64_t o) {
