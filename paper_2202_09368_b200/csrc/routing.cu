@@ -177,9 +177,17 @@ size_t topk_scratch_bytes(int64_t n, int E, int64_t k) { return topk_layout(n, E
 
 __device__ __forceinline__ int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
-// Walks the [t0, t1) x [c0, c0 + cw) slab of S with every thread of the CTA and calls f(score, token,
-// column within the chunk).  VEC: 16-byte loads (E a multiple of 4), else scalar.  Four independent
-// loads per thread are in flight.
+// Walks the [t0, t1) x [c0, c0 + cw) slab of S with every thread of the CTA.  A thread always sees the same
+// columns (four consecutive ones with VEC, one without): slab_first_col() tells it which, or -1 for none,
+// and f(score, token, j) gets the j-th of them, j a compile-time 0..3, so per-column state can sit in
+// registers.  VEC: 16-byte loads (E a multiple of 4), else scalar.  Four independent loads per thread
+// are in flight.
+template <bool VEC>
+__device__ __forceinline__ int slab_first_col(int cw) {
+  const int lane = threadIdx.x & 31;
+  if constexpr (VEC) { const int lpr = pow2_at_least((cw + 3) >> 2); const int g = (lane % lpr) * 4; return g < cw ? g : -1; }
+  else { const int cwp = pow2_at_least(cw); const int cc = lane % cwp; return cc < cw ? cc : -1; }
+}
 template <bool VEC, typename F>
 __device__ __forceinline__ void for_slab(const float* __restrict__ S, int E, int c0, int cw, int64_t t0, int64_t t1, F&& f) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -198,7 +206,7 @@ __device__ __forceinline__ void for_slab(const float* __restrict__ S, int E, int
       for (int u = 0; u < U; ++u)
         if (t + u * step < t1) {
           const int64_t tt = t + u * step;
-          f(v[u].x, tt, g); f(v[u].y, tt, g + 1); f(v[u].z, tt, g + 2); f(v[u].w, tt, g + 3);
+          f(v[u].x, tt, 0); f(v[u].y, tt, 1); f(v[u].z, tt, 2); f(v[u].w, tt, 3);
         }
     }
   } else {
@@ -213,7 +221,7 @@ __device__ __forceinline__ void for_slab(const float* __restrict__ S, int E, int
         if (t + u * step < t1) v[u] = S[(t + u * step) * E + c0 + cc];
 #pragma unroll
       for (int u = 0; u < U; ++u)
-        if (t + u * step < t1) f(v[u], t + u * step, cc);
+        if (t + u * step < t1) f(v[u], t + u * step, 0);
     }
   }
 }
@@ -245,12 +253,23 @@ topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int 
   const int shift = 52 - kRadixBits * pass;            // score bits 29..20, 19..10, 9..0
   const int64_t t0 = (int64_t)blockIdx.x * rows_per_cta;
   const int64_t t1 = min(n, t0 + rows_per_cta);
-  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
-    if (!s_active[col]) return;
-    const unsigned long long key = make_key(s, t);
-    const bool match = pass == 0 || ((key ^ s_prefix[col]) >> (shift + kRadixBits)) == 0;
-    if (match) atomicAdd(&sh[(unsigned)((key >> shift) & (kBins - 1)) * kTopkChunk + col], 1u);
-  });
+  {
+    // only the score half of the key matters here: v = ~bits(S), digit (v >> sh32) & 1023, and from the
+    // second pass on the bits above the digit have to equal the expert's prefix
+    constexpr int NC = VEC ? 4 : 1;
+    const int col0 = slab_first_col<VEC>(cw), sh32 = shift - 32;
+    bool act[NC]; unsigned want[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+      act[j] = col0 >= 0 && col0 + j < cw && s_active[col0 + j];
+      want[j] = act[j] ? (unsigned)(s_prefix[col0 + j] >> 32) >> (sh32 + kRadixBits) : 0u;
+    }
+    for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t, int j) {
+      const unsigned v = ~__float_as_uint(s);
+      if (act[j] && (pass == 0 || (v >> (sh32 + kRadixBits)) == want[j]))
+        atomicAdd(&sh[((v >> sh32) & (kBins - 1)) * kTopkChunk + col0 + j], 1u);
+    });
+  }
   __syncthreads();
   for (int i = tid; i < kBins * kTopkChunk; i += kHistThreads) {
     const unsigned v = sh[i];
@@ -371,13 +390,25 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
     if (kind == 0) { if (pos < k) keys[(size_t)(c0 + col) * kpad + pos] = key; }
     else if (pos < (unsigned)kCandCap) cand[(size_t)(c0 + col) * kCandCap + pos] = key;
   };
-  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int col) {
-    const unsigned long long key = make_key(s, t), hi = key >> s_shift[col];
-    int kind;                                          // mode 3: the tie walk has placed the keys at the threshold
-    if (hi < s_thr[col]) kind = 0;
-    else if (hi == s_thr[col] && s_mode[col] == 1) kind = 0;
-    else if (hi == s_thr[col] && s_mode[col] == 2) kind = 1;
-    else return;
+  // per column of this thread: the decided score bits (thr, after dropping the low bits of v = ~bits(S) that
+  // are still open) and what happens to a key exactly at the threshold: 0 winner, 1 candidate, 2 nothing
+  // (the tie walk has placed it)
+  constexpr int NC = VEC ? 4 : 1;
+  const int col0 = slab_first_col<VEC>(cw);
+  unsigned thr[NC], drop[NC]; int at_thr[NC];
+#pragma unroll
+  for (int j = 0; j < NC; ++j) {
+    const bool ok = col0 >= 0 && col0 + j < cw;
+    drop[j] = ok ? s_shift[col0 + j] - 32 : 0; thr[j] = ok ? (unsigned)s_thr[col0 + j] : 0u;
+    at_thr[j] = !ok ? 2 : (s_mode[col0 + j] == 1 ? 0 : (s_mode[col0 + j] == 2 ? 1 : 2));
+  }
+  for_slab<VEC>(S, E, c0, cw, t0, t1, [&](float s, int64_t t, int j) {
+    const unsigned hi = ~__float_as_uint(s) >> drop[j];
+    if (hi > thr[j]) return;
+    const int kind = hi < thr[j] ? 0 : at_thr[j];
+    if (kind == 2) return;
+    const int col = col0 + j;
+    const unsigned long long key = make_key(s, t);
     const unsigned idx = atomicAdd(&s_n, 1u);
     if (idx < (unsigned)kCompactCap) { s_key[idx] = key; s_tag[idx] = (unsigned char)(col | (kind << 7)); }
     else put(kind, col, atomicAdd(&cursor[kind * E + c0 + col], 1u), key);
@@ -526,8 +557,9 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I,
                : cudaFuncSetAttribute(topk_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSmemBytes)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(base, 0, L.zero_bytes, st)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(keys, 0xFF, (size_t)E * L.kpad * 8, st)) != cudaSuccess) return e;
-  // rows per CTA: about two CTAs per SM over all chunks, at least 256 rows each
-  int64_t want = (int64_t)148 * 2 / L.chunks; if (want < 1) want = 1;
+  // rows per CTA: one CTA per SM fits (the histogram takes 132 KiB of shared memory), so one wave over all
+  // chunks; at least 256 rows each
+  int64_t want = (int64_t)148 / L.chunks; if (want < 1) want = 1;
   int64_t rows = (n + want - 1) / want; if (rows < 256) rows = 256;
   const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks);
   for (int pass = 0; pass < kRadixPasses; ++pass) {
