@@ -100,6 +100,18 @@ def workload_desc(name):
             f"one routing group per GPU")
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
+# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 634.3 MB at 4 experts of
+# the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
+# moves E/4 times as much.  None for shapes that were not captured.
+GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 634.3e6 / 4, "cfg4e4": 634.3e6 / 4}
+
+
+def gemm_traffic(workload, E):
+    per = GEMM_TRAFFIC_PER_EXPERT.get(workload)
+    return None if per is None else per * E
+
+
 def layer_flops(n, d, dff, E, c):
     slots = int(n * c)
     gemm = 2.0 * slots * d * dff                 # one expert-batched GEMM
@@ -304,7 +316,7 @@ def run_gpu(args):
                                                       "and their backward)",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": (achieved / peak) if achieved else None,
-                         "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": None,
+                         "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": gemm_traffic(args.workload, E),
                          "flops_per_launch": fl["gemm"], "avg_launch_ms": gemm_avg_ms},
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
             "layer_tflops": (fl["fwd"] + fl["bwd"]) / (ms_step * 1e-3) / 1e12,
