@@ -94,10 +94,11 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def workload_desc(name):
+def workload_desc(name, groups=1):
     n, d, dff, E, c = WORKLOADS[name]
+    how = "one routing group per GPU" if groups == 1 else f"{groups} routing groups of {n // groups} tokens per GPU"
     return (f"{name}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} fwd+bwd, bf16 storage / fp32 accumulate, "
-            f"one routing group per GPU")
+            f"{how}")
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
@@ -120,7 +121,7 @@ def layer_flops(n, d, dff, E, c):
 
 
 # ----------------------------------------------------------------------------------- CPU oracle timing
-def time_oracle_sample(n, d, dff, E, c, seed=0, budget_s=12.0):
+def time_oracle_sample(n, d, dff, E, c, seed=0, budget_s=12.0, groups=1):
     """Times the oracle on routing in full plus as many whole experts forward + backward as fit in
     about `budget_s` seconds of CPU work (at least one, at most E) and extrapolates the expert part
     to E experts.  Returns (tokens/s, threads, description)."""
@@ -144,7 +145,7 @@ def time_oracle_sample(n, d, dff, E, c, seed=0, budget_s=12.0):
         return w.float().numpy().astype(np.float64).reshape(d, dff)
 
     t0 = time.perf_counter()
-    r = O.route(X, Wg, c)
+    r = O.route(X, Wg, c, groups=groups)
     t_route = time.perf_counter() - t0
     t_sum, experts = 0.0, 0
     while experts < E and (experts == 0 or t_route + t_sum < budget_s):
@@ -174,13 +175,13 @@ def run_reference(args):
         return
     vals = []
     for _ in range(max(1, min(args.steps, 2))):          # bounded: each step is seconds of CPU work
-        v, threads, what = time_oracle_sample(n, d, dff, E, c)
+        v, threads, what = time_oracle_sample(n, d, dff, E, c, groups=args.groups)
         vals.append(v)
     v = sum(vals) / len(vals)
     out = {"impl": "reference", "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": v, "unit": "tokens/s",
            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / v,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": workload_desc(args.workload)},
+           "config": {"workload": workload_desc(args.workload, args.groups)},
            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -213,7 +214,8 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)
     n, d, dff, E, c = WORKLOADS[args.workload]
     bf = torch.bfloat16
-    cfg = B.make_config(n, d, dff, E, c, bf)
+    assert n % args.groups == 0
+    cfg = B.make_config(n // args.groups, d, dff, E, c, bf, groups=args.groups)
     seed = rank                                                   # each rank routes its own group
     chunk = 1 << 26
     X = IN.normal_tensor((n, d), 1.0, seed, IN.TID_X, bf, dev, chunk)
@@ -298,13 +300,13 @@ def run_gpu(args):
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            v, threads, what = time_oracle_sample(n, d, dff, E, c)
+            v, threads, what = time_oracle_sample(n, d, dff, E, c, groups=args.groups)
             cpu = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what}
         out = {
             "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": world * n / (ms_step * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_desc(args.workload),
+            "config": {"workload": workload_desc(args.workload, args.groups),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
                              if args.workload != "small" else "small case, L2 resident",
                        "tensor_cores": bool(B.ec_uses_tensor_cores(cfg))},
@@ -406,6 +408,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' instead of the grid")
     args = ap.parse_args()

@@ -8,6 +8,16 @@
  * factor c, k = n*c/e tokens per expert (Eq. 1).  A "slot" is one (expert i,
  * position j) pair; its flat id is i*k + j and there are e*k of them.
  *
+ * Routing groups.  The paper routes one group of n tokens (Section 3.2) and names, under
+ * Limitations, routing several groups independently as the way to use the method where a
+ * token must not compete with all others (for example, tokens of one sequence spread over
+ * groups).  cfg->groups = g > 1 does that: X holds g*n rows, group r being rows r*n ..
+ * r*n + n - 1 (how tokens are assigned to groups is the caller's arrangement of X); every
+ * expert takes the top k = n*c/e tokens of each group, so it serves g*k slots.  In every
+ * shape below read then n as g*n (rows of X, S, X_out, row_ptr) and k as g*k (row length of
+ * I and G, slots per expert), with an expert's slots ordered by group and, inside a group,
+ * as for one group; token indices are global row numbers of X.  g = 1 is the paper's layer.
+ *
  * Conventions for every entry point unless it says otherwise
  *  - Tensor arguments are DEVICE pointers owned by the caller, dense row-major,
  *    16-byte aligned.  The library never allocates, frees or keeps device memory.
@@ -22,7 +32,8 @@
  *  - X, Wg, W1, W2, X_out, dX_out and all gradients have the element type
  *    cfg->dtype; S, G and X_e are always fp32 and index outputs are int32.
  *  - Restrictions (EC_ERR_UNSUPPORTED otherwise): d_model and d_ff rows must be a
- *    multiple of 16 bytes long; n < 2^31; 1 <= E <= 256; E*k < 2^31; groups == 1.
+ *    multiple of 16 bytes long; groups*n < 2^31; 1 <= E <= 256; E*groups*k < 2^31;
+ *    1 <= groups <= 65535.
  */
 #ifndef ECMOE_H_
 #define ECMOE_H_
@@ -52,7 +63,7 @@ typedef struct {
   int32_t d_model; /* d                                                               */
   int32_t d_ff;    /* d'                                                              */
   int32_t E;       /* number of experts e                                             */
-  int32_t groups;  /* independent routing groups; must be 1                           */
+  int32_t groups;  /* independent routing groups of n tokens each, >= 1 (see above)       */
   double c;        /* capacity factor (Eq. 1)                                         */
   int32_t dtype;   /* ec_dtype                                                        */
   int32_t gelu;    /* ec_gelu                                                         */
@@ -71,7 +82,7 @@ typedef struct {
   float* X_e;       /* [E, k, d]  expert outputs H[i] . W2[i]^T, fp32 on both paths    */
 } ec_saved_ptrs;
 
-/* Eq. 1: k = floor(n*c/E).  Returns -1 when cfg is NULL or k falls outside [1, n]. */
+/* Eq. 1: k = floor(n*c/E), per routing group.  Returns -1 when cfg is NULL or k falls outside [1, n]. */
 int64_t ec_capacity(const ec_config* cfg);
 
 /* Bytes of scratch every call below needs (the maximum over the three).  0 on a bad cfg. */

@@ -128,19 +128,29 @@ def expert_ffn_backward(dX_e_i, X_in_i, Z_i, H_i, W1_i, W2_i, gelu_variant: str 
     return dW1, dW2, dX_in, dH, dZ
 
 
-def route(X, Wg, c: float, S_override=None):
-    """Eq. 1-2: S, G, I and the token->slot inverse index."""
-    n = np.asarray(X).shape[0]
+def route(X, Wg, c: float, S_override=None, groups: int = 1):
+    """Eq. 1-2: S, G, I and the token->slot inverse index.
+
+    groups > 1 (the paper's Limitations section: route several groups of tokens independently):
+    X holds `groups` blocks of n rows; Eq. 1-2 are applied to each block on its own with k = n*c/e,
+    and expert i's row of I and G lists its k tokens of group 0, then of group 1, ...; token
+    indices are row numbers of X.  k in the result is then groups * (n*c/e)."""
+    N = np.asarray(X).shape[0]
     e = np.asarray(Wg).shape[1]
+    if N % groups:
+        raise ValueError("rows of X must divide into the groups")
+    n = N // groups
     k = capacity(n, c, e)
     S = gate(X, Wg) if S_override is None else np.asarray(S_override, F64)
-    G, I = topk(S, k)
-    row_ptr, slots = inverse_index(I, n)
-    return dict(k=k, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots)
+    parts = [topk(S[g * n:(g + 1) * n], k) for g in range(groups)]
+    G = np.concatenate([p[0] for p in parts], axis=1)
+    I = np.concatenate([p[1] + g * n for g, p in enumerate(parts)], axis=1)
+    row_ptr, slots = inverse_index(I, N)
+    return dict(k=k * groups, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots)
 
 
 def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
-            store=_keep):
+            store=_keep, groups: int = 1):
     """Eq. 1-4.  Returns every intermediate.
 
     S_override replaces the gate output (the routing is then taken from it);
@@ -156,7 +166,7 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
     W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
     n, d = X.shape
     e = Wg.shape[1]
-    r = route(X, Wg, c, S_override)
+    r = route(X, Wg, c, S_override, groups)
     k, S = r["k"], r["S"]
     if I_override is not None:
         I = np.asarray(I_override, np.int64)

@@ -88,7 +88,16 @@ def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=
 
 
 def ec_capacity(cfg: ec_config) -> int:
+    """Eq. 1 per routing group."""
     return int(lib().ec_capacity(C.byref(cfg)))
+
+
+def total_tokens(cfg: ec_config) -> int:
+    return cfg.n * cfg.groups
+
+
+def slots_per_expert(cfg: ec_config) -> int:
+    return ec_capacity(cfg) * cfg.groups
 
 
 def ec_workspace_bytes(cfg: ec_config) -> int:
@@ -145,15 +154,15 @@ class Routing:
 
 def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
     """Eq. 1-2 on device tensors; returns S, I, G and the token->slot index."""
-    k = ec_capacity(cfg)
-    if k < 1:
+    if ec_capacity(cfg) < 1:
         raise EcError(EC_ERR_INVALID_ARG, "ec_capacity")
+    n, k = total_tokens(cfg), slots_per_expert(cfg)
     dev = X.device
     if out is None:
-        out = Routing(torch.empty(cfg.n, cfg.E, dtype=torch.float32, device=dev),
+        out = Routing(torch.empty(n, cfg.E, dtype=torch.float32, device=dev),
                       torch.empty(cfg.E, k, dtype=torch.int32, device=dev),
                       torch.empty(cfg.E, k, dtype=torch.float32, device=dev),
-                      torch.empty(cfg.n + 1, dtype=torch.int32, device=dev),
+                      torch.empty(n + 1, dtype=torch.int32, device=dev),
                       torch.empty(cfg.E * k, dtype=torch.int32, device=dev))
     ws = alloc_workspace(cfg, dev) if ws is None else ws
     _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
@@ -163,7 +172,7 @@ def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
 
 def ec_shuffle(cfg, X, I, X_in=None):
     """Eq. 3 shuffle: X_in[i, j, :] = X[I[i, j], :]."""
-    k = ec_capacity(cfg)
+    k = slots_per_expert(cfg)
     if X_in is None:
         X_in = torch.empty(cfg.E, k, cfg.d_model, dtype=X.dtype, device=X.device)
     _check(lib().ec_shuffle(C.byref(cfg), _ptr(X), _ptr(I), _ptr(X_in), _stream()), "ec_shuffle")
@@ -173,7 +182,7 @@ def ec_shuffle(cfg, X, I, X_in=None):
 def ec_unshuffle(cfg, X_e, G, row_ptr, slots, X_out=None):
     """Eq. 4 unshuffle: X_out[t, :] = sum over the slots of t of G[s] * X_e[s, :] (X_e, G fp32)."""
     if X_out is None:
-        X_out = torch.empty(cfg.n, cfg.d_model, dtype=_torch_dtype(cfg), device=X_e.device)
+        X_out = torch.empty(total_tokens(cfg), cfg.d_model, dtype=_torch_dtype(cfg), device=X_e.device)
     _check(lib().ec_unshuffle(C.byref(cfg), _ptr(X_e), _ptr(G), _ptr(row_ptr), _ptr(slots), _ptr(X_out), _stream()),
            "ec_unshuffle")
     return X_out
@@ -196,7 +205,7 @@ def ec_route_static(cfg, X, Wg, out: Routing) -> Routing:
 def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None):
     """Eq. 2-4.  Returns (X_out, saved)."""
     dev = X.device
-    X_out = torch.empty(cfg.n, cfg.d_model, dtype=_torch_dtype(cfg), device=dev) if X_out is None else X_out
+    X_out = torch.empty(total_tokens(cfg), cfg.d_model, dtype=_torch_dtype(cfg), device=dev) if X_out is None else X_out
     saved = alloc_saved(cfg, dev) if saved is None else saved
     ws = alloc_workspace(cfg, dev) if ws is None else ws
     _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),
@@ -243,7 +252,7 @@ def saved_view(cfg, saved) -> dict:
     """Torch views of the parts of the forward->backward blob (no copies)."""
     v = ec_saved_ptrs()
     _check(lib().ec_saved_view(C.byref(cfg), _ptr(saved), C.byref(v)), "ec_saved_view")
-    k = ec_capacity(cfg)
+    k = slots_per_expert(cfg)
     base = saved.data_ptr()
     dt = _torch_dtype(cfg)
     es = 4 if cfg.dtype == EC_F32 else 2
@@ -255,7 +264,7 @@ def saved_view(cfg, saved) -> dict:
         off = addr - base
         return saved[off:off + cnt * esz].view(dtype).view(*shape)
 
-    n, E, d, f = cfg.n, cfg.E, cfg.d_model, cfg.d_ff
+    n, E, d, f = total_tokens(cfg), cfg.E, cfg.d_model, cfg.d_ff
     return dict(S=view(v.S, (n, E), torch.float32, 4), I=view(v.I, (E, k), torch.int32, 4),
                 G=view(v.G, (E, k), torch.float32, 4), row_ptr=view(v.row_ptr, (n + 1,), torch.int32, 4),
                 slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es),

@@ -16,21 +16,24 @@ constexpr size_t kAlign = 256;
 inline size_t up(size_t b) { return (b + kAlign - 1) & ~(kAlign - 1); }
 inline size_t esize(int dtype) { return dtype == EC_F32 ? 4 : 2; }
 
-struct Dims { int64_t n, k, slots; int d, dff, E; int dtype, gelu; size_t eb; };
+// n: all tokens of the call (groups * tokens per group), k: slots per expert (groups * k per group),
+// slots = E * k; ng, kg: the per-group values Eq. 1 is about.
+struct Dims { int64_t n, k, slots, ng, kg; int d, dff, E, groups; int dtype, gelu; size_t eb; };
 
 ec_status check_cfg(const ec_config* c, Dims* D) {
   if (!c) return EC_ERR_INVALID_ARG;
   if (c->dtype != EC_F32 && c->dtype != EC_BF16) return EC_ERR_INVALID_ARG;
   if (c->gelu != EC_GELU_ERF && c->gelu != EC_GELU_TANH) return EC_ERR_INVALID_ARG;
   if (c->n < 1 || c->d_model < 1 || c->d_ff < 1 || c->E < 1 || !(c->c > 0.0)) return EC_ERR_INVALID_ARG;
-  if (c->groups != 1) return EC_ERR_UNSUPPORTED;
-  if (c->n >= ((int64_t)1 << 31) || c->E > 256) return EC_ERR_UNSUPPORTED;
+  if (c->groups < 1) return EC_ERR_INVALID_ARG;
+  if (c->n * c->groups >= ((int64_t)1 << 31) || c->E > 256 || c->groups > 65535) return EC_ERR_UNSUPPORTED;
   const size_t eb = esize(c->dtype);
   if ((c->d_model * eb) % 16 || (c->d_ff * eb) % 16) return EC_ERR_UNSUPPORTED;
   const int64_t k = ec_capacity(c);
   if (k < 1) return EC_ERR_INVALID_ARG;
-  if ((int64_t)c->E * k >= ((int64_t)1 << 31)) return EC_ERR_UNSUPPORTED;
-  if (D) { D->n = c->n; D->k = k; D->slots = (int64_t)c->E * k; D->d = c->d_model; D->dff = c->d_ff;
+  if ((int64_t)c->E * k * c->groups >= ((int64_t)1 << 31)) return EC_ERR_UNSUPPORTED;
+  if (D) { D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
+           D->slots = (int64_t)c->E * D->k; D->d = c->d_model; D->dff = c->d_ff;
            D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb; }
   return EC_OK;
 }
@@ -68,7 +71,7 @@ WsLayout ws_layout(const Dims& D) {
   auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
   L.status = take(sizeof(StatusWord));
   const size_t base = o;
-  L.topk = take(topk_scratch_bytes(D.n, D.E, D.k));
+  L.topk = take(topk_scratch_bytes(D.ng, D.E, D.kg, D.groups));
   L.inverse = take(inverse_scratch_bytes(D.n));
   const size_t fwd_end = o;
   o = base;                                   // the backward pass reuses the same region
@@ -161,7 +164,7 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
   }
   if (!done) EC_CUDA(launch_gate_softmax_simt(D.dtype, X, Wg, S, D.n, D.d, D.E, st));
   prof_mark("gate_softmax", st);
-  EC_CUDA(launch_topk(S, D.n, D.E, D.k, I, G, ws + W.topk, st));
+  EC_CUDA(launch_topk(S, D.ng, D.E, D.kg, D.groups, I, G, ws + W.topk, st));
   prof_mark("topk", st);
   EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
   prof_mark("inverse_index", st);

@@ -33,8 +33,10 @@ void count_launch(int n = 1);
 cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, float* S, int64_t n,
                                      int d, int E, cudaStream_t st);
 // scratch layout for the selection is described in routing.cu; bytes needed:
-size_t topk_scratch_bytes(int64_t n, int E, int64_t k);
-cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I, float* G,
+// `groups` independent routing groups of n tokens each (S has groups * n rows); I and G are [E, groups * k],
+// group g of an expert at positions g * k .. g * k + k - 1, with global token indices
+size_t topk_scratch_bytes(int64_t n, int E, int64_t k, int groups);
+cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups, int32_t* I, float* G,
                         void* scratch, cudaStream_t st);
 size_t inverse_scratch_bytes(int64_t n);
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t slots_total, int32_t* row_ptr,

@@ -157,23 +157,25 @@ struct TopkLayout {
   size_t off_state, off_hist, off_counters, off_cursor, off_cand, off_keys, zero_bytes, total;
   int chunks; int64_t kpad;
 };
-static TopkLayout topk_layout(int64_t n, int E, int64_t k) {
+// E experts of each of `groups` routing groups: groups * E independent columns ("virtual experts", group-major)
+static TopkLayout topk_layout(int64_t n, int E, int64_t k, int groups) {
   TopkLayout L;
   L.chunks = (E + kTopkChunk - 1) / kTopkChunk;
+  const size_t VE = (size_t)groups * E;
   L.kpad = 1; while (L.kpad < k) L.kpad <<= 1;
   size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += (b + 255) & ~(size_t)255; return r; };
-  L.off_state = take(sizeof(SelState) * (size_t)E);
-  L.off_hist = take((size_t)E * kBins * 4);
-  L.off_counters = take((size_t)kRadixPasses * L.chunks * 4);
-  L.off_cursor = take((size_t)2 * E * 4);
+  L.off_state = take(sizeof(SelState) * VE);
+  L.off_hist = take(VE * kBins * 4);
+  L.off_counters = take((size_t)kRadixPasses * groups * L.chunks * 4);
+  L.off_cursor = take(2 * VE * 4);
   L.zero_bytes = o;                       // everything up to here starts at zero
-  L.off_cand = take((size_t)E * kCandCap * 8);
-  L.off_keys = take((size_t)E * L.kpad * 8);
+  L.off_cand = take(VE * kCandCap * 8);
+  L.off_keys = take(VE * L.kpad * 8);
   L.total = o;
   return L;
 }
-size_t topk_scratch_bytes(int64_t n, int E, int64_t k) { return topk_layout(n, E, k).total; }
+size_t topk_scratch_bytes(int64_t n, int E, int64_t k, int groups) { return topk_layout(n, E, k, groups).total; }
 
 __device__ __forceinline__ int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
@@ -234,8 +236,10 @@ topk_hist_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int 
   __shared__ unsigned long long s_prefix[kTopkChunk];
   __shared__ int s_active[kTopkChunk];
   __shared__ int s_any, s_last;
-  const int tid = threadIdx.x, chunk = blockIdx.y, nchunks = gridDim.y;
+  const int tid = threadIdx.x, chunk = blockIdx.y, nchunks = gridDim.y, grp = blockIdx.z;
   const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
+  S += (size_t)grp * n * E;                            // this group's n rows; its experts' state, histograms
+  state += (size_t)grp * E; hist += (size_t)grp * E * kBins; counters += (size_t)grp * kRadixPasses * nchunks;
   if (tid == 0) s_any = 0;
   __syncthreads();
   if (tid < kTopkChunk) {
@@ -331,7 +335,8 @@ topk_ties_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, int6
                  unsigned long long* keys) {
   __shared__ unsigned s_warp[32];
   __shared__ unsigned s_total;
-  const int e = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int e = blockIdx.x, grp = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  S += (size_t)grp * n * E; state += (size_t)grp * E; keys += (size_t)grp * E * kpad;
   if (state[e].mode != 0) return;
   const unsigned thr = (unsigned)(state[e].prefix >> 32), k_rem = state[e].k_rem, k_def = k - k_rem;
   unsigned running = 0;
@@ -373,8 +378,12 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
   __shared__ unsigned s_cnt[2][kTopkChunk], s_base[2][kTopkChunk], s_n;
   __shared__ unsigned long long s_thr[kTopkChunk];
   __shared__ unsigned s_shift[kTopkChunk], s_mode[kTopkChunk];
-  const int tid = threadIdx.x, chunk = blockIdx.y;
+  const int tid = threadIdx.x, chunk = blockIdx.y, grp = blockIdx.z, groups = gridDim.z;
   const int c0 = chunk * kTopkChunk, cw = min(kTopkChunk, E - c0);
+  S += (size_t)grp * n * E; state += (size_t)grp * E;
+  keys += (size_t)grp * E * kpad; cand += (size_t)grp * E * kCandCap;
+  unsigned* cursor_w = cursor + (size_t)grp * E;                       // winners; candidates follow all groups' winners
+  unsigned* cursor_c = cursor + (size_t)groups * E + (size_t)grp * E;
   if (tid == 0) s_n = 0;
   if (tid < kTopkChunk) {
     s_cnt[0][tid] = s_cnt[1][tid] = 0;
@@ -411,7 +420,7 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
     const unsigned long long key = make_key(s, t);
     const unsigned idx = atomicAdd(&s_n, 1u);
     if (idx < (unsigned)kCompactCap) { s_key[idx] = key; s_tag[idx] = (unsigned char)(col | (kind << 7)); }
-    else put(kind, col, atomicAdd(&cursor[kind * E + c0 + col], 1u), key);
+    else put(kind, col, atomicAdd(&(kind ? cursor_c : cursor_w)[c0 + col], 1u), key);
   });
   __syncthreads();
   const int held = (int)min(s_n, (unsigned)kCompactCap);
@@ -419,7 +428,7 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
   __syncthreads();
   if (tid < 2 * kTopkChunk) {
     const int w = tid / kTopkChunk, col = tid % kTopkChunk;
-    if (col < cw) { const unsigned c = s_cnt[w][col]; s_base[w][col] = c ? atomicAdd(&cursor[w * E + c0 + col], c) : 0u; }
+    if (col < cw) { const unsigned c = s_cnt[w][col]; s_base[w][col] = c ? atomicAdd(&(w ? cursor_c : cursor_w)[c0 + col], c) : 0u; }
   }
   __syncthreads();
   if (tid < kTopkChunk) s_cnt[0][tid] = s_cnt[1][tid] = 0;
@@ -430,8 +439,13 @@ topk_compact_kernel(const float* __restrict__ S, int64_t n, int E, unsigned k, i
   }
 }
 
-__device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, float* G, int64_t o) {
-  I[o] = (int32_t)(unsigned)(key & 0xFFFFFFFFull);
+// Slot j of virtual expert ve = group * E + expert lands in row `expert` of I and G (each groups * k long) at
+// position group * k + j, and the token index becomes global (group * n + token within the group).
+struct SlotMap { int E, groups; int64_t k, n; };
+__device__ __forceinline__ void emit_slot(unsigned long long key, int32_t* I, float* G, const SlotMap& m, int64_t ve, int64_t j) {
+  const int64_t grp = ve / m.E, e = ve % m.E;
+  const int64_t o = (e * m.groups + grp) * m.k + j;
+  I[o] = (int32_t)((unsigned)(key & 0xFFFFFFFFull) + (unsigned)(grp * m.n));
   G[o] = __uint_as_float(~(unsigned)(key >> 32));
 }
 
@@ -463,7 +477,7 @@ __device__ __forceinline__ void load_sorted_candidates(const unsigned long long*
 constexpr int kSortThreads = 1024;
 __global__ void __launch_bounds__(kSortThreads)
 topk_finish_tile_kernel(const unsigned long long* __restrict__ keys, const unsigned long long* __restrict__ cand,
-                        const SelState* __restrict__ state, int64_t kpad, int64_t k, int32_t* I, float* G) {
+                        const SelState* __restrict__ state, int64_t kpad, int64_t k, SlotMap map, int32_t* I, float* G) {
   __shared__ unsigned long long sk[kSortTile];
   __shared__ unsigned long long sc[kCandCap];
   const int e = blockIdx.x;
@@ -477,7 +491,7 @@ topk_finish_tile_kernel(const unsigned long long* __restrict__ keys, const unsig
     __syncthreads();
   }
   bitonic_smem(sk, (int)kpad);
-  for (int i = threadIdx.x; i < k; i += kSortThreads) emit_slot(sk[i], I, G, (int64_t)e * k + i);
+  for (int i = threadIdx.x; i < k; i += kSortThreads) emit_slot(sk[i], I, G, map, e, i);
 }
 
 // k beyond one tile: the candidates are merged into the global key list first.
@@ -497,7 +511,7 @@ topk_resolve_kernel(unsigned long long* keys, const unsigned long long* __restri
 // size_lo..size_hi (powers of two); for a size larger than the tile only the strides that fit.
 __global__ void __launch_bounds__(kSortThreads)
 topk_sort_tile_kernel(unsigned long long* keys, int64_t kpad, int64_t k, int64_t size_lo, int64_t size_hi,
-                      int emit, int32_t* I, float* G) {
+                      int emit, SlotMap map, int32_t* I, float* G) {
   __shared__ unsigned long long sk[kSortTile];
   const int64_t tiles_per_expert = (kpad + kSortTile - 1) / kSortTile;
   const int64_t expert = blockIdx.x / tiles_per_expert;
@@ -520,7 +534,7 @@ topk_sort_tile_kernel(unsigned long long* keys, int64_t kpad, int64_t k, int64_t
   }
   if (emit) {
     for (int i = threadIdx.x; i < len; i += kSortThreads)
-      if (base + i < k) emit_slot(sk[i], I, G, expert * k + base + i);
+      if (base + i < k) emit_slot(sk[i], I, G, map, expert, base + i);
   } else {
     for (int i = threadIdx.x; i < len; i += kSortThreads) src[i] = sk[i];
   }
@@ -540,9 +554,10 @@ __global__ void topk_sort_global_kernel(unsigned long long* keys, int64_t kpad, 
   }
 }
 
-cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I, float* G,
+cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups, int32_t* I, float* G,
                         void* scratch, cudaStream_t st) {
-  const TopkLayout L = topk_layout(n, E, k);
+  const TopkLayout L = topk_layout(n, E, k, groups);
+  const int64_t VE = (int64_t)groups * E;              // independent columns: E per group
   char* base = (char*)scratch;
   SelState* state = (SelState*)(base + L.off_state);
   unsigned* hist = (unsigned*)(base + L.off_hist);
@@ -550,46 +565,47 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int32_t* I,
   unsigned* cursor = (unsigned*)(base + L.off_cursor);
   unsigned long long* cand = (unsigned long long*)(base + L.off_cand);
   unsigned long long* keys = (unsigned long long*)(base + L.off_keys);
+  const SlotMap map = {E, groups, k, n};
   cudaError_t e;
   const bool vec = E % 4 == 0 && ((uintptr_t)S & 15) == 0;
-  // the histogram kernels use 128 KiB of dynamic shared memory
+  // the histogram kernels use 132 KiB of dynamic shared memory
   if ((e = vec ? cudaFuncSetAttribute(topk_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSmemBytes)
                : cudaFuncSetAttribute(topk_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHistSmemBytes)) != cudaSuccess) return e;
   if ((e = cudaMemsetAsync(base, 0, L.zero_bytes, st)) != cudaSuccess) return e;
-  if ((e = cudaMemsetAsync(keys, 0xFF, (size_t)E * L.kpad * 8, st)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(keys, 0xFF, (size_t)VE * L.kpad * 8, st)) != cudaSuccess) return e;
   // rows per CTA: one CTA per SM fits (the histogram takes 132 KiB of shared memory), so one wave over all
-  // chunks; at least 256 rows each
-  int64_t want = (int64_t)148 / L.chunks; if (want < 1) want = 1;
+  // chunks and groups; at least 256 rows each
+  int64_t want = (int64_t)148 / ((int64_t)L.chunks * groups); if (want < 1) want = 1;
   int64_t rows = (n + want - 1) / want; if (rows < 256) rows = 256;
-  const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks);
+  const dim3 grid((unsigned)((n + rows - 1) / rows), (unsigned)L.chunks, (unsigned)groups);
   for (int pass = 0; pass < kRadixPasses; ++pass) {
     count_launch();
     if (vec) topk_hist_kernel<true><<<grid, kHistThreads, kHistSmemBytes, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
     else topk_hist_kernel<false><<<grid, kHistThreads, kHistSmemBytes, st>>>(S, n, E, (unsigned)k, pass, (int)rows, state, hist, counters);
   }
   count_launch();
-  topk_ties_kernel<<<E, 1024, 0, st>>>(S, n, E, (unsigned)k, L.kpad, state, keys);
+  topk_ties_kernel<<<dim3(E, groups), 1024, 0, st>>>(S, n, E, (unsigned)k, L.kpad, state, keys);
   count_launch();
   if (vec) topk_compact_kernel<true><<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys, cand);
   else topk_compact_kernel<false><<<grid, kHistThreads, 0, st>>>(S, n, E, (unsigned)k, L.kpad, (int)rows, state, cursor, keys, cand);
   if (L.kpad <= kSortTile) {
     count_launch();
-    topk_finish_tile_kernel<<<E, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k, I, G);
+    topk_finish_tile_kernel<<<(unsigned)VE, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k, map, I, G);
   } else {
     const int64_t tiles = (L.kpad + kSortTile - 1) / kSortTile;
-    const unsigned sort_grid = (unsigned)(E * tiles);
+    const unsigned sort_grid = (unsigned)(VE * tiles);
     count_launch();
-    topk_resolve_kernel<<<E, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k);
+    topk_resolve_kernel<<<(unsigned)VE, kSortThreads, 0, st>>>(keys, cand, state, L.kpad, k);
     count_launch();
-    topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, kSortTile, 0, I, G);
-    const int64_t pairs = (int64_t)E * (L.kpad >> 1);
+    topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, 2, kSortTile, 0, map, I, G);
+    const int64_t pairs = VE * (L.kpad >> 1);
     for (int64_t size = 2 * kSortTile; size <= L.kpad; size <<= 1) {
       for (int64_t stride = size >> 1; stride >= kSortTile; stride >>= 1) {
         count_launch();
         topk_sort_global_kernel<<<grid_for(pairs, 256), 256, 0, st>>>(keys, L.kpad, pairs, size, stride);
       }
       count_launch();
-      topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, size, size, size == L.kpad, I, G);
+      topk_sort_tile_kernel<<<sort_grid, kSortThreads, 0, st>>>(keys, L.kpad, k, size, size, size == L.kpad, map, I, G);
     }
   }
   return cudaGetLastError();
@@ -749,13 +765,24 @@ __global__ void combine_kernel(const float* __restrict__ X_e, const float* __res
     const int64_t t = g / quads_per_row; const int v = (int)(g % quads_per_row);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const int a = row_ptr[t], b = row_ptr[t + 1];
-    for (int q = a; q < b; ++q) {
-      const int s = slots[q];
-      const float w = G[s];
-      float x[4];
-      load4(X_e + ((int64_t)s * quads_per_row + v) * 4, x);
+    // four slots at a time: their ids, then their weights and row pieces, are fetched together, and
+    // added in slot order
+    for (int q0 = a; q0 < b; q0 += 4) {
+      int s[4]; float w[4]; float4 x[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) acc[i] = fmaf(w, x[i], acc[i]);
+      for (int u = 0; u < 4; ++u) s[u] = q0 + u < b ? slots[q0 + u] : -1;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        w[u] = s[u] >= 0 ? G[s[u]] : 0.f;
+        x[u] = s[u] >= 0 ? *reinterpret_cast<const float4*>(X_e + ((int64_t)s[u] * quads_per_row + v) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (s[u] >= 0) {
+          acc[0] = fmaf(w[u], x[u].x, acc[0]); acc[1] = fmaf(w[u], x[u].y, acc[1]);
+          acc[2] = fmaf(w[u], x[u].z, acc[2]); acc[3] = fmaf(w[u], x[u].w, acc[3]);
+        }
+      }
     }
     store4(X_out + g * 4, acc);
   }

@@ -49,22 +49,25 @@ def to_np(t):
 
 def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
     """Step (ii): bit-exact routing given the GPU's own S."""
-    k = B.ec_capacity(cfg)
+    k, n, g = B.ec_capacity(cfg), cfg.n, cfg.groups
     S32 = S_gpu.cpu().numpy()                      # float32 bits, compared as such
-    G_ref, I_ref = O.topk(S32, k)
+    parts = [O.topk(S32[r * n:(r + 1) * n], k) for r in range(g)]          # every routing group on its own
+    G_ref = np.concatenate([p[0] for p in parts], axis=1)
+    I_ref = np.concatenate([p[1] + r * n for r, p in enumerate(parts)], axis=1)
     I_np = I_gpu.cpu().numpy()
     assert np.array_equal(I_np, I_ref), f"I differs in {(I_np != I_ref).sum()} of {I_ref.size} slots"
     assert np.array_equal(G_gpu.cpu().numpy().view(np.uint32), G_ref.view(np.uint32))
-    rp_ref, sl_ref = O.inverse_index(I_ref, cfg.n)
+    rp_ref, sl_ref = O.inverse_index(I_ref, n * g)
     assert np.array_equal(row_ptr.cpu().numpy(), rp_ref)
     assert np.array_equal(slots.cpu().numpy(), sl_ref)
     return I_ref
 
 
-def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True):
-    """Runs forward (+ backward) on the GPU and checks every tensor against the oracle."""
+def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1):
+    """Runs forward (+ backward) on the GPU and checks every tensor against the oracle.
+    n is the number of tokens per routing group; li holds groups * n rows."""
     tol = TOL[dtype]
-    cfg = B.make_config(n, d, dff, E, c, dtype, gelu)
+    cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups)
     dev = "cuda"
     X, Wg, W1, W2 = (t.to(dev) for t in (li.X, li.Wg, li.W1, li.W2))
     ws = B.alloc_workspace(cfg)
@@ -77,7 +80,7 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         errs["S"] = rel_err(to_np(v["S"]), O.gate(Xn, Wgn))
         assert errs["S"] <= tol, errs
     check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
-    f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy())
+    f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(), groups=groups)
     assert np.array_equal(v["X_in"].float().cpu().numpy(), Xn[f["I"]].astype(np.float32))   # gather is a copy
     for name in ("Z", "H", "X_e"):
         errs[name] = rel_err(to_np(v[name]), f[name])
@@ -94,7 +97,7 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
     bound = {k_: tol for k_ in errs}
     if dtype == torch.bfloat16:
         ff = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(),
-                       store=bf16_store)
+                       store=bf16_store, groups=groups)
         floor = {k_: rel_err(ff[k_], f[k_]) for k_ in ("Z", "H", "X_e", "X_out")}
         if backward:
             fb = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), ff, gelu, store=bf16_store)

@@ -62,3 +62,31 @@ def test_capacity_factor_sweep_forward(c, scale):
     errs = run_and_check(n, d, dff, E, c, BF16, li, backward=False)
     assert B.ec_capacity(B.make_config(n, d, dff, E, c, BF16)) == int(n * c / E)
     print(c, scale, {k_: (f"{v:.3e}" if not isinstance(v, dict) else v) for k_, v in errs.items()})
+
+
+@pytest.mark.parametrize("dtype,groups,n,d,dff,E,c", [
+    (torch.float32, 3, 100, 24, 40, 5, 1.5),       # ragged, E not a multiple of 4: scalar top-k path
+    (torch.float32, 2, 256, 64, 128, 8, 2.0),
+    (BF16, 4, 512, 128, 256, 16, 2.0),             # k = 64 per group, 256 slots per expert: two-CTA GEMMs
+    (BF16, 8, 1024, 256, 512, 64, 1.0),            # 16 tokens per expert and group
+])
+def test_routing_groups_forward_backward(dtype, groups, n, d, dff, E, c):
+    """Several routing groups per call (the Limitations section's suggestion): each block of n rows is routed
+    on its own, experts serve groups * k slots."""
+    li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=4)
+    run_and_check(n, d, dff, E, c, dtype, li, groups=groups)
+
+
+def test_routing_groups_match_separate_calls():
+    """Routing g groups in one call selects, group by group, what g separate one-group calls select."""
+    groups, n, d, E, c = 4, 2048, 128, 32, 2.0
+    li = IN.make_layer_inputs(groups * n, d, 8, E, BF16, seed=6, with_grad=False)
+    X, Wg = li.X.cuda(), li.Wg.cuda()
+    many = B.ec_route(B.make_config(n, d, 8, E, c, BF16, groups=groups), X, Wg)
+    one_cfg = B.make_config(n, d, 8, E, c, BF16)
+    k = B.ec_capacity(one_cfg)
+    for g in range(groups):
+        one = B.ec_route(one_cfg, X[g * n:(g + 1) * n], Wg)
+        assert torch.equal(many.S[g * n:(g + 1) * n], one.S)
+        assert torch.equal(many.I[:, g * k:(g + 1) * k], one.I + g * n)
+        assert torch.equal(many.G[:, g * k:(g + 1) * k], one.G)

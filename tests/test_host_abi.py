@@ -44,7 +44,9 @@ def test_sizes_and_rejections():
     k = 128
     assert B.ec_saved_bytes(cfg) >= 4 * (256 * 4 + 3 * 4 * k + 257) + 4 * 4 * k * (2 * 64 + 2 * 256)
     assert B.ec_workspace_bytes(cfg) > 0
-    assert B.ec_workspace_bytes(B.make_config(256, 64, 256, 4, 2.0, groups=2)) == 0
+    assert B.ec_workspace_bytes(B.make_config(256, 64, 256, 4, 2.0, groups=0)) == 0
+    two = B.make_config(256, 64, 256, 4, 2.0, groups=2)                            # two routing groups: twice the rows and slots
+    assert B.ec_capacity(two) == k and B.ec_saved_bytes(two) >= 2 * 4 * (256 * 4 + 3 * 4 * k) + 2 * 4 * 4 * k * (2 * 64 + 2 * 256)
     assert B.ec_workspace_bytes(B.make_config(256, 63, 256, 4, 2.0)) == 0          # rows not 16-byte multiples
     assert B.ec_workspace_bytes(B.make_config(256, 64, 256, 300, 2.0)) == 0        # E > 256
     big = B.make_config(16384, 4096, 16384, 64, 2.0, torch.bfloat16)

@@ -259,3 +259,46 @@ def test_backward_gate_gradient_is_orthogonal_to_constant_logit_shift():
     f = O.forward(X, Wg, W1, W2, 2.0)
     b = O.backward(X, Wg, W1, W2, R, f)
     np.testing.assert_allclose(b["dL"].sum(axis=1), 0.0, atol=1e-12)
+
+
+# ---------------------------------------------------------------- routing groups (Limitations section)
+@pytest.mark.parametrize("groups,n,E,c", [(2, 24, 4, 2.0), (3, 16, 2, 1.0), (4, 10, 5, 1.5)])
+def test_routing_groups_are_independent_layers_on_the_blocks(groups, n, E, c):
+    """Experts act on rows independently, so routing g groups separately must give, on every block of n rows,
+    exactly what the (already pinned) one-group layer gives on that block alone; the index lists are those of
+    the blocks shifted to global row numbers, and every expert holds k tokens of every group."""
+    d, dff = 6, 10
+    X, Wg, W1, W2, R = mk(groups * n, d, dff, E, seed=11)
+    f = O.forward(X, Wg, W1, W2, c, groups=groups)
+    k = O.capacity(n, c, E)
+    assert f["I"].shape == (E, groups * k) and f["k"] == groups * k
+    for g in range(groups):
+        blk = slice(g * n, (g + 1) * n)
+        one = O.forward(X[blk], Wg, W1, W2, c)
+        assert np.array_equal(f["I"][:, g * k:(g + 1) * k], one["I"] + g * n)
+        assert np.array_equal(f["G"][:, g * k:(g + 1) * k], one["G"])
+        np.testing.assert_allclose(f["X_out"][blk], one["X_out"], rtol=0, atol=1e-13)
+        for i in range(E):                              # k distinct tokens of this group per expert
+            own = f["I"][i, g * k:(g + 1) * k]
+            assert len(set(own.tolist())) == k and own.min() >= g * n and own.max() < (g + 1) * n
+    cnt = O.experts_per_token(f["row_ptr"])
+    assert cnt.sum() == int(groups * n * c)
+    assert np.array_equal(O.route(X, Wg, c, groups=1)["I"], O.route(X, Wg, c)["I"])     # one group: the paper's layer
+    # the backward pass on grouped routing against finite differences (I frozen)
+    b = O.backward(X, Wg, W1, W2, R, f)
+    rng = np.random.default_rng(3)
+    h = 1e-6
+
+    def loss(Xp, Wgp, W1p, W2p):
+        gq = O.forward(Xp, Wgp, W1p, W2p, c, groups=groups)
+        assert np.array_equal(gq["I"], f["I"])
+        return float((R * gq["X_out"]).sum())
+
+    for name, idx in (("dX", 0), ("dWg", 1), ("dW1", 2), ("dW2", 3)):
+        base = [X, Wg, W1, W2]
+        D = rng.standard_normal(base[idx].shape)
+        plus = list(base); plus[idx] = base[idx] + h * D
+        minus = list(base); minus[idx] = base[idx] - h * D
+        fd = (loss(*plus) - loss(*minus)) / (2 * h)
+        an = float((b[name] * D).sum())
+        assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (name, fd, an)
