@@ -34,6 +34,9 @@ WORKLOADS = {
     "cfg4": (16384, 4096, 16384, 64, 2.0),      # 8B/64E-shaped layer (headline)
     "cfg2": (8192, 768, 3072, 32, 2.0),         # 100M/32E-shaped layer
     "cfg4e4": (1024, 4096, 16384, 4, 2.0),      # four experts of the 8B/64E shape (profiling-sized)
+    "cfg3c05": (8192, 768, 3072, 64, 0.5),      # capacity-factor sweep, 100M/64E shape: k = 64
+    "cfg3c1": (8192, 768, 3072, 64, 1.0),       #   k = 128
+    "cfg3c2": (8192, 768, 3072, 64, 2.0),       #   k = 256
     "small": (2048, 256, 512, 8, 2.0),
 }
 GEMM_STAGES = ("gemm1_gelu", "gemm2", "gemm_dZ", "gemm_dW2", "gemm_dW1", "gemm_dXin")
@@ -356,7 +359,11 @@ def run_routing(args):
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     dev = torch.device("cuda")
     d, c, bf = 1024, 2.0, torch.bfloat16
-    grid = ROUTING_GRID if not args.route_case else [tuple(int(v) for v in args.route_case.split(","))]
+    grid = ROUTING_GRID
+    if args.route_case:                                   # "n,E" or "n,E,d"
+        vals = [int(v) for v in args.route_case.split(",")]
+        grid = [tuple(vals[:2])]
+        d = vals[2] if len(vals) > 2 else d
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     peaks = measured_peaks()
     cases = []
@@ -389,7 +396,7 @@ def run_routing(args):
             st[k_] = {"us": round(med * 1e3, 2), "GBps": round(by[k_] / (med * 1e-3) / 1e9, 1),
                       "frac_hbm": round(by[k_] / (med * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
         total_us = sum(v["us"] for v in st.values())
-        cases.append({"n": n, "E": E, "k": int(n * c / E), "stages": st, "chain_us": round(total_us, 2),
+        cases.append({"n": n, "E": E, "d": d, "k": int(n * c / E), "stages": st, "chain_us": round(total_us, 2),
                       "chain_GBps": round(sum(by.values()) / (total_us * 1e-6) / 1e9, 1),
                       "tokens_per_s": round(n / (total_us * 1e-6))})
         del X, Wg, ws, r, X_in, X_e, X_out
@@ -410,7 +417,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
-    ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' instead of the grid")
+    ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")
     args = ap.parse_args()
     if args.routing:
         run_routing(args)
