@@ -37,6 +37,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <mutex>
+#include <type_traits>
 #include <string.h>
 
 namespace ecmoe {
@@ -501,14 +502,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               // both buffers are written: Z into the first, H = GeLU(Z) into the second
               if (lane == 0) bulk_wait_read<0>();
               __syncwarp();
+              // one uniform branch on the GeLU form around the whole chunk: inside it only that form is evaluated
+              auto convert = [&](auto variant) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float z[8], h[8];
+                for (int j = 0; j < 8; ++j) {
+                  float z[8], h[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[8 * j + e]); h[e] = p.gelu == 0 ? gelu_fwd<0>(z[e]) : gelu_fwd<1>(z[e]); }
-                *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ sw) << 4)) = pack8(z);
-                *reinterpret_cast<uint4*>(stg + 4096 + lane * 128 + ((j ^ sw) << 4)) = pack8(h);
-              }
+                  for (int e = 0; e < 8; ++e) { z[e] = __uint_as_float(r[8 * j + e]); h[e] = gelu_fwd<decltype(variant)::value>(z[e]); }
+                  *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ sw) << 4)) = pack8(z);
+                  *reinterpret_cast<uint4*>(stg + 4096 + lane * 128 + ((j ^ sw) << 4)) = pack8(h);
+                }
+              };
+              if (p.gelu == 0) convert(std::integral_constant<int, 0>{}); else convert(std::integral_constant<int, 1>{});
               fence_async_smem();
               __syncwarp();
               if (lane == 0 && r0 < p.M) {
@@ -520,20 +525,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               if constexpr (EPI == EPI_GELU_GRAD) {
                 // dZ = acc * GeLU'(Z): this thread's 64 values of Z (128 bytes of its row)
                 const bf16* zp = p.Zin + obase + n0 + c0;
+                uint4 zv[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                  uint4 zv = make_uint4(0, 0, 0, 0);
-                  if (row_ok && n0 + c0 + 8 * j < p.N) zv = *reinterpret_cast<const uint4*>(zp + 8 * j);
-                  const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w};
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    const float z0 = __uint_as_float(zw[e] << 16), z1 = __uint_as_float(zw[e] & 0xFFFF0000u);
-                    const float g0 = p.gelu == 0 ? gelu_bwd<0>(z0) : gelu_bwd<1>(z0);
-                    const float g1 = p.gelu == 0 ? gelu_bwd<0>(z1) : gelu_bwd<1>(z1);
-                    r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) * g0);
-                    r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) * g1);
-                  }
+                  zv[j] = make_uint4(0, 0, 0, 0);
+                  if (row_ok && n0 + c0 + 8 * j < p.N) zv[j] = *reinterpret_cast<const uint4*>(zp + 8 * j);
                 }
+                auto scale = [&](auto variant) {             // one uniform branch on the GeLU form, as above
+#pragma unroll
+                  for (int j = 0; j < 8; ++j) {
+                    const unsigned zw[4] = {zv[j].x, zv[j].y, zv[j].z, zv[j].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      const float g0 = gelu_bwd<decltype(variant)::value>(__uint_as_float(zw[e] << 16));
+                      const float g1 = gelu_bwd<decltype(variant)::value>(__uint_as_float(zw[e] & 0xFFFF0000u));
+                      r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) * g0);
+                      r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) * g1);
+                    }
+                  }
+                };
+                if (p.gelu == 0) scale(std::integral_constant<int, 0>{}); else scale(std::integral_constant<int, 1>{});
               }
               if constexpr (EPI == EPI_ADD_SLOTS) {
                 // this thread's row gains the rows of its slots (128 bytes of each), in slot order
