@@ -554,9 +554,96 @@ __global__ void topk_sort_global_kernel(unsigned long long* keys, int64_t kpad, 
   }
 }
 
+// Small groups (n <= kSmallN tokens, k <= kSortTile): the whole selection of one expert in one CTA.  The
+// column is brought into shared memory once (as v = ~bits(S)), three 10-bit histogram passes over it find
+// the value of the k-th key exactly, keys below it are winners, keys equal to it win in token order, and the
+// k keys are sorted and written out: one launch instead of eight, for the sizes where launches are what costs.
+constexpr int kSmallN = 16384;
+__global__ void __launch_bounds__(1024)
+topk_small_kernel(const float* __restrict__ S, int n, int E, int k, int kpad, SlotMap map, int32_t* I, float* G) {
+  extern __shared__ unsigned long long sm_keys[];      // [kpad] keys, then [n] values, then [kBins] histogram
+  unsigned* val = reinterpret_cast<unsigned*>(sm_keys + kpad);
+  unsigned* hist = val + n;
+  __shared__ unsigned s_prefix, s_rem, s_less, s_eqtaken, s_warp[33];
+  const int e = blockIdx.x, grp = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* col = S + (size_t)grp * n * E + e;
+  for (int t = tid; t < n; t += 1024) val[t] = ~__float_as_uint(col[(size_t)t * E]);
+  for (int i = tid; i < kpad; i += 1024) sm_keys[i] = ~0ull;
+  if (tid == 0) { s_prefix = 0; s_rem = (unsigned)k; s_less = 0; s_eqtaken = 0; }
+  __syncthreads();
+  // v has its two top bits set (0 <= S <= 1); digits of 10 bits from bit 29 down
+  for (int pass = 0; pass < 3; ++pass) {
+    const int sh = 20 - 10 * pass;
+    for (int i = tid; i < kBins; i += 1024) hist[i] = 0;
+    __syncthreads();
+    const unsigned pre = s_prefix;
+    for (int t = tid; t < n; t += 1024) {
+      const unsigned v = val[t];
+      if (pass == 0 || (v >> (sh + 10)) == (pre >> (sh + 10))) atomicAdd(&hist[(v >> sh) & (kBins - 1)], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {                                   // bucket of the s_rem-th smallest v among the matching ones
+      unsigned c[kBins / 32], lsum = 0;
+#pragma unroll
+      for (int j = 0; j < kBins / 32; ++j) { c[j] = hist[lane * (kBins / 32) + j]; lsum += c[j]; }
+      unsigned incl = lsum;
+      for (int o = 1; o < 32; o <<= 1) { const unsigned u = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += u; }
+      const unsigned excl = incl - lsum, rem = s_rem;
+      if (excl < rem && rem <= incl) {
+        unsigned before = excl; int D = 0;
+#pragma unroll
+        for (int j = 0; j < kBins / 32; ++j) {
+          if (before < rem && rem <= before + c[j]) { D = j; break; }
+          before += c[j];
+        }
+        s_prefix = (pass == 0 ? 0xC0000000u : pre) | ((unsigned)(lane * (kBins / 32) + D) << sh);
+        s_rem = rem - before;
+      }
+    }
+    __syncthreads();
+  }
+  const unsigned thr = s_prefix, k_rem = s_rem, k_less = (unsigned)k - k_rem;      // k_rem keys equal to thr are wanted
+  // winners strictly below the threshold: any order
+  for (int t = tid; t < n; t += 1024)
+    if (val[t] < thr) sm_keys[atomicAdd(&s_less, 1u)] = ((unsigned long long)val[t] << 32) | (unsigned)t;
+  // keys at the threshold: the first k_rem in token order
+  unsigned running = 0;
+  for (int base = 0; base < n && running < k_rem; base += 1024) {
+    const int t = base + tid;
+    const bool m = t < n && val[t] == thr;
+    const unsigned bal = __ballot_sync(0xffffffffu, m);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      const unsigned v = s_warp[lane];
+      unsigned inc = v;
+      for (int o = 1; o < 32; o <<= 1) { const unsigned u = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += u; }
+      s_warp[lane] = inc - v;
+      if (lane == 31) s_warp[32] = inc;
+    }
+    __syncthreads();
+    const unsigned idx = running + s_warp[warp] + __popc(bal & ((1u << lane) - 1u));
+    if (m && idx < k_rem) sm_keys[k_less + idx] = ((unsigned long long)thr << 32) | (unsigned)t;
+    running += s_warp[32];
+    __syncthreads();
+  }
+  __syncthreads();
+  bitonic_smem(sm_keys, kpad);
+  for (int i = tid; i < k; i += 1024) emit_slot(sm_keys[i], I, G, map, (int64_t)grp * E + e, i);
+}
+
 cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups, int32_t* I, float* G,
                         void* scratch, cudaStream_t st) {
   const TopkLayout L = topk_layout(n, E, k, groups);
+  if (n <= kSmallN && L.kpad <= kSortTile) {
+    const SlotMap smap = {E, groups, k, n};
+    const int smem = (int)(L.kpad * 8 + n * 4 + kBins * 4);
+    cudaError_t e0 = cudaFuncSetAttribute(topk_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e0 != cudaSuccess) return e0;
+    count_launch();
+    topk_small_kernel<<<dim3(E, groups), 1024, smem, st>>>(S, (int)n, E, (int)k, (int)L.kpad, smap, I, G);
+    return cudaGetLastError();
+  }
   const int64_t VE = (int64_t)groups * E;              // independent columns: E per group
   char* base = (char*)scratch;
   SelState* state = (SelState*)(base + L.off_state);
