@@ -784,8 +784,51 @@ __global__ void inv_sort_kernel(const int32_t* __restrict__ row_ptr, int64_t n, 
   }
 }
 
+// Small inputs (n <= kInvSmallN tokens, at most kInvSmallSlots slots): the whole inverse index in one CTA and one
+// launch.  Counts and cursors live in shared memory; the order in which atomics hand out places does not
+// matter because every token's list is sorted at the end.
+constexpr int kInvSmallN = 4096, kInvSmallSlots = 1 << 14;
+__global__ void __launch_bounds__(1024)
+inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots) {
+  extern __shared__ int s_cnt[];                       // [n] counts, then cursors
+  __shared__ int s_warp[33];
+  const int tid = threadIdx.x;
+  for (int t = tid; t < n; t += 1024) s_cnt[t] = 0;
+  __syncthreads();
+  for (int s = tid; s < total; s += 1024) atomicAdd(&s_cnt[I[s]], 1);
+  __syncthreads();
+  // exclusive scan over the tokens, 1024 * per at a time
+  const int per = (n + 1023) / 1024, a = min(n, tid * per), b = min(n, a + per);
+  int sum = 0;
+  for (int t = a; t < b; ++t) sum += s_cnt[t];
+  int total_sum;
+  int run = block_exclusive_scan(sum, s_warp, total_sum);
+  for (int t = a; t < b; ++t) { const int c = s_cnt[t]; row_ptr[t] = run; s_cnt[t] = run; run += c; }   // s_cnt becomes the cursor
+  if (tid == 0) row_ptr[n] = total_sum;
+  __syncthreads();
+  for (int s = tid; s < total; s += 1024) slots[atomicAdd(&s_cnt[I[s]], 1)] = s;
+  __syncthreads();
+  __threadfence_block();
+  for (int t = tid; t < n; t += 1024) {                // after the fill s_cnt[t] is the end of token t's list
+    const int lo = t == 0 ? 0 : s_cnt[t - 1], hi = s_cnt[t];
+    for (int i = lo + 1; i < hi; ++i) {
+      const int v = slots[i]; int j = i - 1;
+      while (j >= lo && slots[j] > v) { slots[j + 1] = slots[j]; --j; }
+      slots[j + 1] = v;
+    }
+  }
+}
+
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int32_t* row_ptr, int32_t* slots,
                                  void* scratch, cudaStream_t st) {
+  if (n <= kInvSmallN && total <= kInvSmallSlots) {
+    const int smem = (int)n * 4;
+    cudaError_t e0 = cudaFuncSetAttribute(inv_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e0 != cudaSuccess) return e0;
+    count_launch();
+    inv_small_kernel<<<1, 1024, smem, st>>>(I, (int)n, (int)total, row_ptr, slots);
+    return cudaGetLastError();
+  }
   int32_t* cnt = (int32_t*)scratch;
   int32_t* tile_sum = (int32_t*)((char*)scratch + inv_cnt_bytes(n));
   const unsigned tiles = (unsigned)((n + kScanTile - 1) / kScanTile);
