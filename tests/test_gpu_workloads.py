@@ -90,3 +90,28 @@ def test_routing_groups_match_separate_calls():
         assert torch.equal(many.S[g * n:(g + 1) * n], one.S)
         assert torch.equal(many.I[:, g * k:(g + 1) * k], one.I + g * n)
         assert torch.equal(many.G[:, g * k:(g + 1) * k], one.G)
+
+
+@pytest.mark.parametrize("groups,n,E,c,dtype", [
+    (2, 32768, 64, 2.0, BF16),                  # groups above the single-CTA size: histogram passes, k = 1024 per group
+    (3, 20000, 8, 2.0, torch.float32),          # k = 5000 per group: candidates merged globally, multi-kernel sort
+    (2, 17000, 12, 0.7, torch.float32),         # ragged k, E a multiple of 4 only
+])
+def test_routing_groups_large_groups(groups, n, E, c, dtype):
+    """Routing groups on the multi-kernel top-k path (more than 16384 tokens per group)."""
+    d = 32
+    li = IN.make_layer_inputs(groups * n, d, 8, E, dtype, seed=8, with_grad=False)
+    cfg = B.make_config(n, d, 8, E, c, dtype, groups=groups)
+    r = B.ec_route(cfg, li.X.cuda(), li.Wg.cuda())
+    assert rel_err(to_np(r.S), O.gate(to_np(li.X), to_np(li.Wg))) <= TOL[dtype]
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+def test_routing_groups_with_ties_on_the_multi_kernel_path():
+    """Few distinct logits and large groups: thousands of exactly equal scores at the threshold of every expert
+    and group, resolved toward the lower token by the walk in token order."""
+    groups, n, d, E = 2, 20000, 16, 8
+    X, Wg = IN.quantised_gate_inputs(groups * n, d, E, 2, torch.float32)
+    cfg = B.make_config(n, d, 16, E, 2.0, torch.float32, groups=groups)
+    r = B.ec_route(cfg, X.cuda(), Wg.cuda())
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
