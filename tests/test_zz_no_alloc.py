@@ -39,9 +39,12 @@ def _same_bits(a, b):
 def test_static_scratch_routing_matches_ec_route_on_consecutive_calls():
     dev = torch.device("cuda")
     # (n, d, E, c, dtype, seed): the second shape has fewer experts and more slots per expert than the
-    # first and the third has ties in every column, so stale histograms, cursors or keys would show
+    # first and the third has ties in every column, so stale histograms, cursors or keys would show; the
+    # last two are large enough for the multi-kernel top-k, whose scratch is what the static array holds
     cases = [(4096, 256, 32, 2.0, torch.bfloat16, 0), (3000, 128, 8, 1.0, torch.float32, 1),
-             (2048, 64, 16, 2.0, torch.float32, 2)]
+             (2048, 64, 16, 2.0, torch.float32, 2),
+             (40000, 64, 32, 2.0, torch.bfloat16, 3),       # above the single-kernel sizes: histograms, cursors and keys
+             (36000, 32, 8, 2.0, torch.float32, 4)]         # live in the static array (k = 9000: multi-kernel sort)
     for rep in range(2):
         for n, d, E, c, dtype, seed in cases:
             cfg = B.make_config(n, d, 4 * d, E, c, dtype)
