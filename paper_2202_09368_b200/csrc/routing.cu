@@ -566,18 +566,19 @@ topk_small_kernel(const float* __restrict__ S, int n, int E, int k, int kpad, Sl
   unsigned* hist = val + n;
   __shared__ unsigned s_prefix, s_rem, s_less, s_eqtaken, s_warp[33];
   const int e = blockIdx.x, grp = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nt = blockDim.x, nwarps = nt >> 5;         // 128 .. 1024 threads, by the size of the group
   const float* col = S + (size_t)grp * n * E + e;
-  for (int t = tid; t < n; t += 1024) val[t] = ~__float_as_uint(col[(size_t)t * E]);
-  for (int i = tid; i < kpad; i += 1024) sm_keys[i] = ~0ull;
+  for (int t = tid; t < n; t += nt) val[t] = ~__float_as_uint(col[(size_t)t * E]);
+  for (int i = tid; i < kpad; i += nt) sm_keys[i] = ~0ull;
   if (tid == 0) { s_prefix = 0; s_rem = (unsigned)k; s_less = 0; s_eqtaken = 0; }
   __syncthreads();
   // v has its two top bits set (0 <= S <= 1); digits of 10 bits from bit 29 down
   for (int pass = 0; pass < 3; ++pass) {
     const int sh = 20 - 10 * pass;
-    for (int i = tid; i < kBins; i += 1024) hist[i] = 0;
+    for (int i = tid; i < kBins; i += nt) hist[i] = 0;
     __syncthreads();
     const unsigned pre = s_prefix;
-    for (int t = tid; t < n; t += 1024) {
+    for (int t = tid; t < n; t += nt) {
       const unsigned v = val[t];
       if (pass == 0 || (v >> (sh + 10)) == (pre >> (sh + 10))) atomicAdd(&hist[(v >> sh) & (kBins - 1)], 1u);
     }
@@ -604,18 +605,18 @@ topk_small_kernel(const float* __restrict__ S, int n, int E, int k, int kpad, Sl
   }
   const unsigned thr = s_prefix, k_rem = s_rem, k_less = (unsigned)k - k_rem;      // k_rem keys equal to thr are wanted
   // winners strictly below the threshold: any order
-  for (int t = tid; t < n; t += 1024)
+  for (int t = tid; t < n; t += nt)
     if (val[t] < thr) sm_keys[atomicAdd(&s_less, 1u)] = ((unsigned long long)val[t] << 32) | (unsigned)t;
   // keys at the threshold: the first k_rem in token order
   unsigned running = 0;
-  for (int base = 0; base < n && running < k_rem; base += 1024) {
+  for (int base = 0; base < n && running < k_rem; base += nt) {
     const int t = base + tid;
     const bool m = t < n && val[t] == thr;
     const unsigned bal = __ballot_sync(0xffffffffu, m);
     if (lane == 0) s_warp[warp] = __popc(bal);
     __syncthreads();
     if (warp == 0) {
-      const unsigned v = s_warp[lane];
+      const unsigned v = lane < nwarps ? s_warp[lane] : 0u;
       unsigned inc = v;
       for (int o = 1; o < 32; o <<= 1) { const unsigned u = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += u; }
       s_warp[lane] = inc - v;
@@ -629,7 +630,7 @@ topk_small_kernel(const float* __restrict__ S, int n, int E, int k, int kpad, Sl
   }
   __syncthreads();
   bitonic_smem(sm_keys, kpad);
-  for (int i = tid; i < k; i += 1024) emit_slot(sm_keys[i], I, G, map, (int64_t)grp * E + e, i);
+  for (int i = tid; i < k; i += nt) emit_slot(sm_keys[i], I, G, map, (int64_t)grp * E + e, i);
 }
 
 cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups, int32_t* I, float* G,
@@ -640,8 +641,10 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups,
     const int smem = (int)(L.kpad * 8 + n * 4 + kBins * 4);
     cudaError_t e0 = cudaFuncSetAttribute(topk_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e0 != cudaSuccess) return e0;
+    int threads = 128;                                 // about eight elements per thread
+    while (threads < 1024 && threads * 8 < n) threads <<= 1;
     count_launch();
-    topk_small_kernel<<<dim3(E, groups), 1024, smem, st>>>(S, (int)n, E, (int)k, (int)L.kpad, smap, I, G);
+    topk_small_kernel<<<dim3(E, groups), threads, smem, st>>>(S, (int)n, E, (int)k, (int)L.kpad, smap, I, G);
     return cudaGetLastError();
   }
   const int64_t VE = (int64_t)groups * E;              // independent columns: E per group
