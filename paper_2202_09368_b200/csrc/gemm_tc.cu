@@ -51,14 +51,19 @@ constexpr int BM = 128, BK = 64, UK = 16;
 constexpr int kEpiWarps = 8;                         // two per TMEM lane quarter, each takes half the columns
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kABytes = BM * BK * 2;                 // 16 KiB
-constexpr int kSmemBudget = 160 * 1024;              // operand stages; the epilogue's staging comes on top
+constexpr int kSmemBudget = 224 * 1024;              // operand stages plus the epilogue's staging
 constexpr int kStagingPerWarp = 8192;                // two 4 KiB buffers of 32 rows x 128 bytes
 constexpr int EPI_STORE_F32 = 5;                     // like EPI_STORE with fp32 output
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
 // bn = rows of B one CTA loads per k-block (BN / CTAS)
 __host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + bn * BK * 2; }
-__host__ __device__ constexpr int num_stages(int bn) { return kSmemBudget / stage_bytes(bn) > 8 ? 8 : kSmemBudget / stage_bytes(bn); }
+// Staging for the epilogue: every warp's when the tile is split between the warp pairs, else (a 64-wide tile with
+// the softmax, drained by the first four warps alone) only theirs, which leaves room for more stages.
+__host__ __device__ constexpr int staging_bytes(int bn_tile, int epi) { return (epi == EPI_SOFTMAX && bn_tile < 128 ? 4 : kEpiWarps) * kStagingPerWarp; }
+__host__ __device__ constexpr int num_stages(int bn, int staging) {
+  return (kSmemBudget - staging) / stage_bytes(bn) > 8 ? 8 : (kSmemBudget - staging) / stage_bytes(bn);
+}
 // Two accumulators of BN columns (a power of two for BN = 64, 128, 256).  A CTA pair takes all 512
 // columns, so both CTAs are certain to get base address 0: one tcgen05.mma writes the same
 // tensor-memory address in both.
@@ -269,14 +274,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   constexpr int BNL = BN / CTAS;                    // rows of B this CTA loads
   constexpr int TM = BM * CTAS;                     // rows of the tile the CTA (pair) works on
   constexpr bool kXchg = EPI == EPI_SOFTMAX && BN >= 128;            // the softmax epilogue's exchange area replaces a stage
-  constexpr int S = num_stages(BNL) - (kXchg ? 1 : 0);
+  constexpr int kStaging = staging_bytes(BN, EPI);
+  constexpr int S = num_stages(BNL, kStaging) - (kXchg ? 1 : 0);
   constexpr int kBBytes = BNL * BK * 2;
   constexpr int kStage = kABytes + kBBytes;
   constexpr int kCols = tmem_cols(BN, CTAS);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]; 256 bytes further on, with kXchg: [2][8 warps][32] float2, int[8]
-  uint64_t* bars = (uint64_t*)(smem + S * kStage + kEpiWarps * kStagingPerWarp);
+  uint64_t* bars = (uint64_t*)(smem + S * kStage + kStaging);
   uint32_t* tmem_slot = (uint32_t*)(bars + 2 * S + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
   const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * S, tfull0 = empty0 + 8 * S, tempty0 = tfull0 + 16;
@@ -290,7 +296,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int b = 0; b < 2; ++b) { mbar_init(tfull0 + 8 * b, 1); mbar_init(tempty0 + 8 * b, CTAS * kEpiWarps); }
     *abort_flag = 0;
     if constexpr (kXchg) {
-      int* published = (int*)(smem + S * kStage + kEpiWarps * kStagingPerWarp + 256 + 2 * kEpiWarps * 32 * 8);
+      int* published = (int*)(smem + S * kStage + kStaging + 256 + 2 * kEpiWarps * 32 * 8);
       for (int w = 0; w < kEpiWarps; ++w) published[w] = 0;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -453,7 +459,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // The partner's (max, sum) comes through a slot in shared memory, one per warp and tile parity, with
           // a per-warp counter of published tiles.  A slot is rewritten two tiles later, which the partner's
           // release of the accumulator (it precedes that tile's MMAs) orders after its read.  The wait is bounded.
-          float2* xch = reinterpret_cast<float2*>(smem + S * kStage + kEpiWarps * kStagingPerWarp + 256);
+          float2* xch = reinterpret_cast<float2*>(smem + S * kStage + kStaging + 256);
           volatile int* published = reinterpret_cast<volatile int*>(xch + 2 * kEpiWarps * 32);
           const int me = warp - 2, partner = me ^ 4;
           xch[((it & 1) * kEpiWarps + me) * 32 + lane] = make_float2(mx, sum);
@@ -685,7 +691,7 @@ template <int BN, int EPI, int CTAS>
 cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tc, const CUtensorMap& tc2,
                        const TcParams& p, cudaStream_t st) {
   // the split softmax trades one operand stage for its exchange area (4 KiB + counters), see the kernel
-  constexpr int smem = num_stages(BN / CTAS) * stage_bytes(BN / CTAS) + kEpiWarps * kStagingPerWarp + 1024 + 256;
+  constexpr int smem = num_stages(BN / CTAS, staging_bytes(BN, EPI)) * stage_bytes(BN / CTAS) + staging_bytes(BN, EPI) + 1024 + 256;
   auto kern = gemm_tc_kernel<BN, EPI, CTAS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
