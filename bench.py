@@ -105,10 +105,10 @@ def workload_desc(name, groups=1):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
-# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.0 MB at 4 experts of
+# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.9 MB at 4 experts of
 # the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
 # moves E/4 times as much.  None for shapes that were not captured.
-GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 635.0e6 / 4, "cfg4e4": 635.0e6 / 4}
+GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 635.9e6 / 4, "cfg4e4": 635.9e6 / 4}
 
 
 def gemm_traffic(workload, E):
