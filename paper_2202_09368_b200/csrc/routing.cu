@@ -3,6 +3,8 @@
 // latency-bound integer / fp32 work; the dense contractions live in gemm_*.cu.
 #include "internal.h"
 
+#include <string.h>
+
 namespace ecmoe {
 
 // ------------------------------------------------------------------------------------------
@@ -822,8 +824,67 @@ inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_p
   }
 }
 
+// Medium inputs (n <= kInvClusterN): one cluster of eight CTAs runs the five steps in one launch, with hardware
+// cluster barriers between them (counts and cursors in global memory, the eight tile sums of the scan read
+// from the other CTAs' shared memory).
+constexpr int kInvClusterN = 16384, kInvClusterSlots = 1 << 17, kInvClusterCtas = 8;
+__device__ __forceinline__ void inv_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__global__ void __launch_bounds__(1024)
+inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots, int32_t* cnt) {
+  __shared__ int s_warp[33];
+  __shared__ int s_tile;                               // sum of this CTA's part of the counts
+  const int tid = threadIdx.x, rank = blockIdx.x, nc = gridDim.x;      // the grid is the one cluster
+  const int gtid = rank * 1024 + tid, gsize = nc * 1024;
+  for (int t = gtid; t < n; t += gsize) cnt[t] = 0;
+  inv_cluster_sync();
+  for (int s = gtid; s < total; s += gsize) atomicAdd(&cnt[I[s]], 1);
+  inv_cluster_sync();
+  // exclusive scan: CTA `rank` takes tokens [lo, hi), a thread `per` consecutive ones of them
+  const int per_cta = (n + nc - 1) / nc, lo = min(n, rank * per_cta), hi = min(n, lo + per_cta);
+  const int per = (per_cta + 1023) / 1024, a = min(hi, lo + tid * per), b = min(hi, a + per);
+  int sum = 0;
+  for (int t = a; t < b; ++t) sum += cnt[t];
+  int tile;
+  int run = block_exclusive_scan(sum, s_warp, tile);
+  if (tid == 0) s_tile = tile;
+  inv_cluster_sync();
+  int before = 0;
+  for (int r = 0; r < rank; ++r) {
+    unsigned remote; int v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((unsigned)__cvta_generic_to_shared(&s_tile)), "r"(r));
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote));
+    before += v;
+  }
+  run += before;
+  for (int t = a; t < b; ++t) { const int c = cnt[t]; row_ptr[t] = run; cnt[t] = run; run += c; }      // cnt becomes the cursor
+  if (rank == nc - 1 && tid == 0) row_ptr[n] = before + tile;
+  inv_cluster_sync();
+  for (int s = gtid; s < total; s += gsize) slots[atomicAdd(&cnt[I[s]], 1)] = s;
+  inv_cluster_sync();
+  for (int t = gtid; t < n; t += gsize) {
+    const int p0 = row_ptr[t], p1 = row_ptr[t + 1];
+    for (int i = p0 + 1; i < p1; ++i) {
+      const int v = slots[i]; int j = i - 1;
+      while (j >= p0 && slots[j] > v) { slots[j + 1] = slots[j]; --j; }
+      slots[j + 1] = v;
+    }
+  }
+}
+
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int32_t* row_ptr, int32_t* slots,
                                  void* scratch, cudaStream_t st) {
+  if (n > kInvSmallN && n <= kInvClusterN && total <= kInvClusterSlots) {
+    cudaLaunchConfig_t cfg; memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(kInvClusterCtas); cfg.blockDim = dim3(1024); cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kInvClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    count_launch();
+    return cudaLaunchKernelEx(&cfg, inv_cluster_kernel, I, (int)n, (int)total, row_ptr, slots, (int32_t*)scratch);
+  }
   if (n <= kInvSmallN && total <= kInvSmallSlots) {
     const int smem = (int)n * 4;
     cudaError_t e0 = cudaFuncSetAttribute(inv_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
