@@ -88,6 +88,10 @@ int64_t ec_capacity(const ec_config* cfg);
 /* Bytes of scratch every call below needs (the maximum over the three).  0 on a bad cfg. */
 size_t ec_workspace_bytes(const ec_config* cfg);
 
+/* Bytes of scratch a forward-only call of ec_moe_forward (saved == NULL) needs: the routing scratch plus every
+ * intermediate of Eq. 2-3 except Z.  0 on a bad cfg. */
+size_t ec_forward_only_workspace_bytes(const ec_config* cfg);
+
 /* Bytes of the blob ec_moe_forward fills for ec_moe_backward.  0 on a bad cfg. */
 size_t ec_saved_bytes(const ec_config* cfg);
 
@@ -173,7 +177,10 @@ ec_status ec_route_static(const ec_config* cfg, const void* X, const void* Wg, f
  * fp32, rounded once.  Rows of tokens that no expert chose are zero.
  *   W1, W2 [E, d, d'] (W2 is applied transposed);  X_out [n, d] out.
  * `saved` (ec_saved_bytes(cfg) bytes, 256-byte aligned) receives what the backward
- * pass needs; it must always be given (the intermediates live there).
+ * pass needs (the intermediates live there).  Forward only (inference): pass saved = NULL
+ * and saved_bytes = 0; the intermediates then live in `ws`, which must hold
+ * ec_forward_only_workspace_bytes(cfg) bytes, and Z = X_in . W1, which only the backward
+ * pass reads, is not written at all.  X_out is the same, bit for bit.
  */
 ec_status ec_moe_forward(const ec_config* cfg, const void* X, const void* Wg, const void* W1,
                          const void* W2, void* X_out, void* saved, size_t saved_bytes, void* ws,

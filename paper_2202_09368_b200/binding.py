@@ -22,7 +22,8 @@ EC_GELU_ERF, EC_GELU_TANH = 0, 1
 EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
-           "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle"]
+           "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
+           "ec_forward_only_workspace_bytes"]
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -54,6 +55,7 @@ def lib():
         L.ec_capacity.restype = C.c_int64; L.ec_capacity.argtypes = [P]
         L.ec_workspace_bytes.restype = C.c_size_t; L.ec_workspace_bytes.argtypes = [P]
         L.ec_saved_bytes.restype = C.c_size_t; L.ec_saved_bytes.argtypes = [P]
+        L.ec_forward_only_workspace_bytes.restype = C.c_size_t; L.ec_forward_only_workspace_bytes.argtypes = [P]
         L.ec_saved_view.restype = C.c_int; L.ec_saved_view.argtypes = [P, V, C.POINTER(ec_saved_ptrs)]
         L.ec_route.restype = C.c_int
         L.ec_route.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V]
@@ -202,10 +204,17 @@ def ec_route_static(cfg, X, Wg, out: Routing) -> Routing:
     return out
 
 
-def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None):
-    """Eq. 2-4.  Returns (X_out, saved)."""
+def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None, forward_only=False):
+    """Eq. 2-4.  Returns (X_out, saved); with forward_only nothing is kept for a backward pass (saved is None)."""
     dev = X.device
     X_out = torch.empty(total_tokens(cfg), cfg.d_model, dtype=_torch_dtype(cfg), device=dev) if X_out is None else X_out
+    if forward_only:
+        nb = int(lib().ec_forward_only_workspace_bytes(C.byref(cfg)))
+        if ws is None or ws.numel() < nb:
+            ws = torch.empty(nb, dtype=torch.uint8, device=dev)
+        _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),
+                                    None, 0, _ptr(ws), ws.numel(), _stream()), "ec_moe_forward")
+        return X_out, None
     saved = alloc_saved(cfg, dev) if saved is None else saved
     ws = alloc_workspace(cfg, dev) if ws is None else ws
     _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),

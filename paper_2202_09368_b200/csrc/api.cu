@@ -39,7 +39,8 @@ ec_status check_cfg(const ec_config* c, Dims* D) {
 }
 
 struct SavedLayout { size_t S, I, G, row_ptr, slots, X_in, Z, H, X_e, total; };
-SavedLayout saved_layout(const Dims& D) {
+// with_z = false: the layout of the same tensors without Z (forward-only calls keep them in the workspace)
+SavedLayout saved_layout(const Dims& D, bool with_z = true) {
   SavedLayout L; size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
   L.S = take((size_t)D.n * D.E * 4);
@@ -48,7 +49,7 @@ SavedLayout saved_layout(const Dims& D) {
   L.row_ptr = take((size_t)(D.n + 1) * 4);
   L.slots = take((size_t)D.slots * 4);
   L.X_in = take((size_t)D.slots * D.d * D.eb);
-  L.Z = take((size_t)D.slots * D.dff * D.eb);
+  L.Z = take(with_z ? (size_t)D.slots * D.dff * D.eb : 0);
   L.H = take((size_t)D.slots * D.dff * D.eb);
   L.X_e = take((size_t)D.slots * D.d * 4);          // fp32 on both paths
   L.total = o;
@@ -65,7 +66,7 @@ int dwg_splits(const Dims& D) {
   return (int)(p < 1 ? 1 : (p > 32 ? 32 : p));
 }
 
-struct WsLayout { size_t status, topk, inverse, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
+struct WsLayout { size_t status, topk, inverse, fwd_end, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
 WsLayout ws_layout(const Dims& D) {
   WsLayout L; size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
@@ -74,6 +75,7 @@ WsLayout ws_layout(const Dims& D) {
   L.topk = take(topk_scratch_bytes(D.ng, D.E, D.kg, D.groups));
   L.inverse = take(inverse_scratch_bytes(D.n));
   const size_t fwd_end = o;
+  L.fwd_end = fwd_end;
   o = base;                                   // the backward pass reuses the same region
   L.dX_e = take((size_t)D.slots * D.d * D.eb);
   L.dG = take((size_t)D.slots * 4);
@@ -216,6 +218,11 @@ size_t ec_workspace_bytes(const ec_config* c) {
   return ws_layout(D).total;
 }
 
+size_t ec_forward_only_workspace_bytes(const ec_config* c) {
+  Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
+  return ws_layout(D).fwd_end + saved_layout(D, false).total;
+}
+
 size_t ec_saved_bytes(const ec_config* c) {
   Dims D; if (check_cfg(c, &D) != EC_OK) return 0;
   return saved_layout(D).total;
@@ -295,16 +302,18 @@ ec_status ec_route_static(const ec_config* c, const void* X, const void* Wg, flo
 ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, const void* W1, const void* W2,
                          void* X_out, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
   Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
-  if (!X || !Wg || !W1 || !W2 || !X_out || !saved || !ws) return EC_ERR_INVALID_ARG;
+  if (!X || !Wg || !W1 || !W2 || !X_out || !ws) return EC_ERR_INVALID_ARG;
+  const bool keep = saved != nullptr;                // else forward only: nothing is kept for a backward pass
+  if (!keep && saved_bytes != 0) return EC_ERR_INVALID_ARG;
   if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(W1, 16) || misaligned(W2, 16) || misaligned(X_out, 16) ||
       misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
-  const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D);
-  if (ws_bytes < W.total || saved_bytes < L.total) return EC_ERR_WORKSPACE;
+  const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D, keep);
+  if (keep ? (ws_bytes < W.total || saved_bytes < L.total) : ws_bytes < W.fwd_end + L.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
-  char* sv = (char*)saved; char* w = (char*)ws;
+  char* w = (char*)ws; char* sv = keep ? (char*)saved : w + W.fwd_end;    // forward only: the intermediates follow the routing scratch
   float* S = (float*)(sv + L.S); int32_t* I = (int32_t*)(sv + L.I); float* G = (float*)(sv + L.G);
   int32_t* row_ptr = (int32_t*)(sv + L.row_ptr); int32_t* slots = (int32_t*)(sv + L.slots);
-  void* X_in = sv + L.X_in; void* Z = sv + L.Z; void* H = sv + L.H; float* X_e = (float*)(sv + L.X_e);
+  void* X_in = sv + L.X_in; void* Z = keep ? sv + L.Z : nullptr; void* H = sv + L.H; float* X_e = (float*)(sv + L.X_e);
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   prof_begin(st, 0);

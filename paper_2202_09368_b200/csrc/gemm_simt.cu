@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
         const TC* rows = (const TC*)g.rows;
         for (int q = g.row_ptr[m]; q < g.row_ptr[m + 1]; ++q) v += ldv(rows, (int64_t)g.slots[q] * g.ld_rows + n);
       }
-      stv(C, o, v);
+      if (g.C) stv(C, o, v);                    // EPI_GELU without C: only GeLU(acc) is wanted
     }
   }
 }

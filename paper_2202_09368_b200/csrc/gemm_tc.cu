@@ -79,6 +79,7 @@ struct TcParams {
   int64_t ldc, batch_c;
   int* status;
   int k_split;                                       // batches are cuts of one product along K
+  int skip_c;                                        // EPI_GELU: only H = GeLU(acc) is stored, the accumulator itself is not
   const int32_t* row_ptr; const int32_t* slots; const bf16* rows; int64_t ld_rows;   // EPI_ADD_SLOTS
 };
 
@@ -554,7 +555,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     z[e] = __uint_as_float(r[8 * j + e]); z[e + 1] = __uint_as_float(r[8 * j + e + 1]);
                     gelu_fwd2<decltype(variant)::value>(z[e], z[e + 1], h[e], h[e + 1]);
                   }
-                  *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ sw) << 4)) = pack8(z);
+                  if (!p.skip_c) *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ sw) << 4)) = pack8(z);
                   *reinterpret_cast<uint4*>(stg + 4096 + lane * 128 + ((j ^ sw) << 4)) = pack8(h);
                 }
               };
@@ -562,7 +563,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               fence_async_smem();
               __syncwarp();
               if (lane == 0 && r0 < p.M) {
-                tma_store_3d(&tmC, stg_s, n0 + c0, r0, b);
+                if (!p.skip_c) tma_store_3d(&tmC, stg_s, n0 + c0, r0, b);
                 tma_store_3d(&tmC2, stg_s + 4096, n0 + c0, r0, b);
                 bulk_commit();
               }
@@ -770,7 +771,8 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   if (g.epi == EPI_SOFTMAX) {
     if (!make_map(&tc, g.S, g.N, g.M, 1, g.ldc, 0, 32, 32, true)) return cudaErrorInvalidValue;
   } else {
-    if (!make_map(&tc, g.C, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, 32, g.c_f32 != 0)) return cudaErrorInvalidValue;
+    const void* cbase = (g.epi == EPI_GELU && !g.C) ? g.C2 : g.C;     // without C its map is never used: any valid one will do
+    if (!make_map(&tc, cbase, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, 32, g.c_f32 != 0)) return cudaErrorInvalidValue;
     if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 64, 32)) return cudaErrorInvalidValue;
   }
   TcParams p;
@@ -780,7 +782,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.gelu = g.gelu;
   p.Zin = (const bf16*)g.Zin;
   p.ldc = g.ldc; p.batch_c = g.batch_c; p.status = g.status;
-  p.k_split = g.k_split;
+  p.k_split = g.k_split; p.skip_c = (g.epi == EPI_GELU && !g.C) ? 1 : 0;
   // Tile order.  Tiles running at the same time are consecutive ones.  Along M (default) they share the B tile,
   // which for the expert FFNs is the weight matrix: it is then read from HBM once.  When the output is larger
   // than the operands (short K: the weight gradients) the tiles run along N instead, so that what is written at

@@ -69,7 +69,7 @@ struct GemmArgs {
   int64_t batch_a, batch_b, batch_c;   // element strides between batches
   int64_t k_limit;                     // if > 0, batch b contracts only min(K, k_limit - b*K) terms (split of a long K)
   int epi, gelu;
-  void* C2;                            // EPI_GELU: receives GeLU(acc) (C receives acc)
+  void* C2;                            // EPI_GELU: receives GeLU(acc) (C receives acc, unless C is null)
   const void* Zin;                     // EPI_GELU_GRAD: C = acc * GeLU'(Zin), same layout and dtype as C
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;  // EPI_ADD_SLOTS
 };
@@ -85,7 +85,8 @@ struct TcGemmArgs {
   int64_t lda, ldb; // elements between consecutive rows of the stored matrices
   int64_t batch_a, batch_b;
   int epi, gelu;    // EPI_STORE / EPI_GELU / EPI_GELU_GRAD, or EPI_SOFTMAX below
-  void* C; void* C2; const void* Zin; int64_t ldc; int64_t batch_c;   // bf16 outputs (C is fp32 when c_f32)
+  void* C; void* C2; const void* Zin; int64_t ldc; int64_t batch_c;   // bf16 outputs (C is fp32 when c_f32);
+                                                                      // EPI_GELU with C null writes only C2 = GeLU(acc)
   int c_f32;
   float* S;         // EPI_SOFTMAX: fp32 row softmax of the N columns, [M, N]
   int* status;      // device status word

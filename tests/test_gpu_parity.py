@@ -110,3 +110,22 @@ def test_argument_errors_are_reported_before_any_launch():
         B.ec_route(cfg, X.view(-1)[1:], Wg, ws=ws)          # misaligned pointer
     assert e.value.code == B.EC_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype,n,d,dff,E,c,groups", [(F32, 300, 36, 100, 3, 1.5, 1), (BF16, 2048, 256, 512, 32, 2.0, 1),
+                                                      (BF16, 512, 128, 256, 16, 2.0, 4)])
+def test_forward_only_gives_the_same_output_without_a_saved_blob(dtype, n, d, dff, E, c, groups):
+    """saved = NULL: the intermediates live in the workspace, Z is never written, X_out is the same bits."""
+    li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=9, with_grad=False)
+    cfg = B.make_config(n, d, dff, E, c, dtype, groups=groups)
+    X, Wg, W1, W2 = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2))
+    Y_train, _ = B.ec_moe_forward(cfg, X, Wg, W1, W2)
+    Y_inf, none = B.ec_moe_forward(cfg, X, Wg, W1, W2, forward_only=True)
+    assert none is None
+    assert torch.equal(Y_train.view(torch.uint8), Y_inf.view(torch.uint8))
+    # a workspace that is too small for the intermediates is refused before anything is launched
+    small = torch.empty(B.ec_workspace_bytes(cfg) // 2 if dff > d else 256, dtype=torch.uint8, device="cuda")
+    code = B.lib().ec_moe_forward(__import__("ctypes").byref(cfg), X.data_ptr(), Wg.data_ptr(), W1.data_ptr(), W2.data_ptr(),
+                                  Y_inf.data_ptr(), None, 0, small.data_ptr(), 256, None)
+    assert code == B.EC_ERR_WORKSPACE
+    torch.cuda.synchronize()
