@@ -2,6 +2,7 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4|cfg2|small] [--impl reference]
   python bench.py --routing [--route-case n,E]      (routing-only stress, one extra JSON line format)
+  python bench.py --sweep                           (capacity-factor sweep of the forward pass)
 
 A step is one forward + backward pass of the whole layer over one group of n tokens
 (routing, gather, expert FFNs, combine, and every backward kernel).  Prints ONE JSON
@@ -105,10 +106,10 @@ def workload_desc(name, groups=1):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
-# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.9 MB at 4 experts of
+# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.2 MB at 4 experts of
 # the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
 # moves E/4 times as much.  None for shapes that were not captured.
-GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 635.9e6 / 4, "cfg4e4": 635.9e6 / 4}
+GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 635.2e6 / 4, "cfg4e4": 635.2e6 / 4}
 
 
 def gemm_traffic(workload, E):
@@ -426,6 +427,69 @@ def run_routing(args):
                       "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cases": cases}))
 
 
+# ----------------------------------------------------------------------------------- capacity-factor sweep
+def run_sweep(args):
+    """Forward pass of the 100M/64E-shaped layer (n=8192, d=768, d'=3072, E=64, bf16) for c in {0.5, 1, 2} and gate
+    logits scaled x1 and x4 (the scale multiplies Wg and varies how unevenly tokens are scored).  Per case: forward
+    time (forward-only call, Z not stored), per-stage times, the expert GEMMs against both rooflines (with k = 64 to
+    256 rows per expert they are bound by reading the 302 MB of W1 or W2, not by the tensor cores), and the histogram
+    of the number of experts per token that the routing produced (the quantity of the paper's Fig. 3)."""
+    import torch
+    from paper_2202_09368_b200 import binding as B
+    from paper_2202_09368_b200 import inputs as IN
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dev = torch.device("cuda")
+    n, d, dff, E, bf = 8192, 768, 3072, 64, torch.bfloat16
+    peaks = measured_peaks()
+    X = IN.normal_tensor((n, d), 1.0, 0, IN.TID_X, bf, dev, 1 << 26)
+    W1 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(d), 0, IN.TID_W1, bf, dev, 1 << 26)
+    W2 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(dff), 0, IN.TID_W2, bf, dev, 1 << 26)
+    Y = torch.empty_like(X)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    cases = []
+    for scale in (1.0, 4.0):
+        Wg = IN.normal_tensor((d, E), scale / math.sqrt(d), 0, IN.TID_WG, bf, dev, 1 << 26)
+        for c in (0.5, 1.0, 2.0):
+            cfg = B.make_config(n, d, dff, E, c, bf)
+            ws = torch.empty(int(B.lib().ec_forward_only_workspace_bytes(__import__("ctypes").byref(cfg))), dtype=torch.uint8, device=dev)
+            reps = max(5, min(args.steps, 30))
+            for _ in range(3):
+                B.ec_moe_forward(cfg, X, Wg, W1, W2, Y, None, ws, forward_only=True)
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            B.ec_profile_enable(True)
+            acc = {}
+            for a, b_ in ev:
+                flush.zero_()                                   # the weights (604 MB) exceed L2 anyway; the activations do not
+                a.record()
+                B.ec_moe_forward(cfg, X, Wg, W1, W2, Y, None, ws, forward_only=True)
+                b_.record()
+                for k_, v_ in B.ec_profile_read():
+                    acc.setdefault(k_, []).append(v_)
+            B.ec_profile_enable(False)
+            torch.cuda.synchronize()
+            ms = sorted(a.elapsed_time(b_) for a, b_ in ev)[reps // 2]
+            st = {k_: round(sorted(v_)[len(v_) // 2], 4) for k_, v_ in acc.items()}
+            r = B.ec_route(cfg, X, Wg)
+            per_token = (r.row_ptr[1:] - r.row_ptr[:-1]).long()
+            hist = torch.bincount(per_token, minlength=1).tolist()
+            k = int(n * c / E)
+            flops = 2.0 * n * c * d * dff                       # one expert GEMM
+            wbytes = E * d * dff * 2
+            gem = {}
+            for g_ in ("gemm1_gelu", "gemm2"):
+                t = st[g_] * 1e-3
+                gem[g_] = {"ms": st[g_], "TFLOPs": round(flops / t / 1e12, 1), "frac_tensor": round(flops / t / 1e12 / peaks["tflops_burst"], 3),
+                           "weight_GBps": round(wbytes / t / 1e9, 1), "frac_hbm": round(wbytes / t / 1e9 / peaks["hbm_gbs"], 3)}
+            cases.append({"c": c, "logit_scale": scale, "k": k, "forward_ms": round(ms, 4), "tokens_per_s": round(n / (ms * 1e-3)),
+                          "stage_ms": st, "expert_gemms": gem, "experts_per_token_hist": hist,
+                          "tokens_without_expert": hist[0], "max_experts_per_token": len(hist) - 1})
+    print(json.dumps({"metric": "ec_moe_forward_capacity_sweep", "unit": "ms (median, forward only)",
+                      "config": {"workload": f"capacity-factor sweep: n={n} d={d} d_ff={dff} E={E} bf16 forward, c x logit scale",
+                                 "l2": "512 MiB flush before every timed call"},
+                      "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_burst": peaks["tflops_burst"], "source": peaks["source"]},
+                      "cases": cases}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -436,9 +500,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
+    ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")
     args = ap.parse_args()
-    if args.routing:
+    if args.sweep:
+        run_sweep(args)
+    elif args.routing:
         run_routing(args)
     elif args.impl == "reference":
         run_reference(args)
