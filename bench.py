@@ -43,6 +43,10 @@ WORKLOADS = {
 GEMM_STAGES = ("gemm1_gelu", "gemm2", "gemm_dZ", "gemm_dW2", "gemm_dW1", "gemm_dXin")
 
 
+# nominal figures the targets are phrased against (context; the measured peaks are the roofline denominators)
+NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -341,6 +345,7 @@ def run_gpu(args):
                                                       "and their backward)",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": (achieved / peak) if achieved else None,
+                         "frac_of_nominal": (achieved / NOMINAL_BF16_TFLOPS) if achieved else None,
                          "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": gemm_traffic(args.workload, E),
                          "flops_per_launch": fl["gemm"], "avg_launch_ms": gemm_avg_ms},
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
@@ -414,7 +419,8 @@ def run_routing(args):
             v_.sort()
             med = v_[len(v_) // 2]
             st[k_] = {"us": round(med * 1e3, 2), "GBps": round(by[k_] / (med * 1e-3) / 1e9, 1),
-                      "frac_hbm": round(by[k_] / (med * 1e-3) / 1e9 / peaks["hbm_gbs"], 3)}
+                      "frac_hbm": round(by[k_] / (med * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+                      "frac_nominal": round(by[k_] / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 3)}
         total_us = sum(v["us"] for v in st.values())
         cases.append({"n": n, "E": E, "d": d, "k": int(n * c / E), "stages": st, "chain_us": round(total_us, 2),
                       "chain_GBps": round(sum(by.values()) / (total_us * 1e-6) / 1e9, 1),
