@@ -684,7 +684,9 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int pick_bn(const TcGemmArgs& g) { return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64); }
+// 256 columns per tile when the tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
+// streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
+int pick_bn(const TcGemmArgs& g) { return (g.N > 128 && g.M > BM) ? 256 : (g.N > 64 ? 128 : 64); }
 // Two CTAs per tile when a tile of 256 rows is not mostly padding and the pair's B halves are whole 64-wide blocks.
 int pick_ctas(const TcGemmArgs& g, int bn) { return (bn >= 128 && g.M > BM) ? 2 : 1; }
 
