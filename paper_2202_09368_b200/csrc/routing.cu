@@ -456,7 +456,7 @@ __device__ __forceinline__ void bitonic_smem(unsigned long long* a, int len) {
   for (int size = 2; size <= len; size <<= 1) {
     for (int stride = size >> 1; stride >= 1; stride >>= 1) {
       for (int p = threadIdx.x; p < (len >> 1); p += blockDim.x) {
-        const int i = (p / stride) * 2 * stride + (p % stride), j = i + stride;
+        const int i = ((p & ~(stride - 1)) << 1) | (p & (stride - 1)), j = i + stride;      // stride is a power of two
         const bool asc = (i & size) == 0;
         const unsigned long long x = a[i], y = a[j];
         if ((x > y) == asc) { a[i] = y; a[j] = x; }
@@ -525,7 +525,7 @@ topk_sort_tile_kernel(unsigned long long* keys, int64_t kpad, int64_t k, int64_t
   for (int64_t size = size_lo; size <= size_hi; size <<= 1) {
     for (int64_t stride = min(size >> 1, (int64_t)(len >> 1)); stride >= 1; stride >>= 1) {
       for (int p = threadIdx.x; p < (len >> 1); p += kSortThreads) {
-        const int i = (int)((p / stride) * 2 * stride + (p % stride));
+        const int i = (int)((((int64_t)p & ~(stride - 1)) << 1) | ((int64_t)p & (stride - 1)));   // stride is a power of two
         const int j = i + (int)stride;
         const bool asc = ((base + i) & size) == 0;
         const unsigned long long a = sk[i], b = sk[j];
@@ -548,7 +548,7 @@ __global__ void topk_sort_global_kernel(unsigned long long* keys, int64_t kpad, 
   for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < total_pairs;
        p += (int64_t)gridDim.x * blockDim.x) {
     const int64_t expert = p / (kpad >> 1), q = p % (kpad >> 1);
-    const int64_t i = (q / stride) * 2 * stride + (q % stride), j = i + stride;
+    const int64_t i = ((q & ~(stride - 1)) << 1) | (q & (stride - 1)), j = i + stride;       // stride is a power of two
     unsigned long long* kk = keys + expert * kpad;
     const bool asc = (i & size) == 0;
     const unsigned long long a = kk[i], b = kk[j];
