@@ -132,6 +132,12 @@ cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, f
 // equal scores a lower token.  Keys of one expert are distinct, so "the k smallest keys, ascending"
 // is the unique answer with ties broken toward the lower token and slots listed by descending score.
 //
+// Routing groups (several independent groups of n tokens) multiply the columns: every (group, expert) pair is
+// selected on its own and lands in its expert's row of I and G at the group's offset.
+//
+// Groups of up to kSmallN tokens with k up to one sort tile take one launch (topk_small_kernel, further down:
+// one CTA per column does everything in shared memory).  Larger ones take the path described next.
+//
 // Selection is a most-significant-digit radix select over the 30 significant score bits, 10 bits a
 // pass, run for all experts at once: a pass histograms its digit of the keys that still match the
 // expert's prefix (in shared memory, merged into one global histogram per expert), and the last
@@ -143,8 +149,8 @@ cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, f
 // one CTA per such expert walks the column in token order and takes the first ones.  One more pass
 // over S then copies the winners (and candidates) out, and a bitonic network sorts each expert's keys.
 //
-// scratch: [SelState E][hist E*1024 u32][counters passes*chunks u32][cursors 2E u32] (zeroed per call)
-//          [candidates E*kCandCap u64][keys E*kpad u64]
+// scratch, with C = groups * E columns: [SelState C][hist C*1024 u32][counters passes*groups*chunks u32]
+//          [cursors 2C u32] (zeroed per call) [candidates C*kCandCap u64][keys C*kpad u64]
 // ------------------------------------------------------------------------------------------
 constexpr int kHistThreads = 1024;
 constexpr int kBins = 1 << kRadixBits;
