@@ -247,6 +247,19 @@ def run_gpu(args):
     for _ in range(max(3, args.warmup)):
         step()
     assert B.ec_read_status(ws) == B.EC_OK
+    if args.graph:
+        # the step as one CUDA graph: the library only queues work on the given stream, so a forward + backward
+        # pair can be captured once and replayed, which takes the launch latencies out of small steps
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.stream(side):
+            step()
+        torch.cuda.current_stream(dev).wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        eager_step, step = step, graph.replay
+        step(); torch.cuda.synchronize()
     # ---- timed region: K steps, device timed, max over ranks
     barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -268,9 +281,10 @@ def run_gpu(args):
     B.ec_profile_enable(True)
     stage_ms = {}
     bursts, burst_steps = 3, max(2, min(args.steps, 10))
+    plain_step = eager_step if args.graph else step         # the stage events are recorded at launch time
     for _ in range(bursts):
         for _ in range(burst_steps):
-            step()
+            plain_step()
         for k_, v_ in B.ec_profile_read():
             stage_ms[k_] = stage_ms.get(k_, 0.0) + v_ / bursts
     B.ec_profile_enable(False)
@@ -336,7 +350,8 @@ def run_gpu(args):
             "config": {"workload": workload_desc(args.workload, args.groups),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
                              if args.workload != "small" else "small case, L2 resident",
-                       "tensor_cores": bool(B.ec_uses_tensor_cores(cfg))},
+                       "tensor_cores": bool(B.ec_uses_tensor_cores(cfg)),
+                       "launch": "one CUDA graph per step" if args.graph else "stream launches"},
             "clocks": clocks.summary(),
             "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": io_bytes,
                     "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms},
@@ -504,6 +519,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="time the step as one captured CUDA graph")
     ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")

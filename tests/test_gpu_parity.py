@@ -129,3 +129,33 @@ def test_forward_only_gives_the_same_output_without_a_saved_blob(dtype, n, d, df
                                   Y_inf.data_ptr(), None, 0, small.data_ptr(), 256, None)
     assert code == B.EC_ERR_WORKSPACE
     torch.cuda.synchronize()
+
+
+def test_a_step_can_be_captured_in_a_cuda_graph():
+    """Forward and backward only queue work on the caller's stream: a step captured once replays to the same bits."""
+    n, d, dff, E = 1024, 128, 256, 8
+    li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=5)
+    cfg = B.make_config(n, d, dff, E, 2.0, BF16)
+    X, Wg, W1, W2, dY = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2, li.dX_out))
+    ws, saved, Y = B.alloc_workspace(cfg), B.alloc_saved(cfg), torch.empty_like(X)
+    grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
+
+    def step():
+        B.ec_moe_forward(cfg, X, Wg, W1, W2, Y, saved, ws)
+        B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, grads, ws)
+
+    step(); torch.cuda.synchronize()
+    want = [t.clone() for t in (Y,) + grads]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (Y,) + grads:
+        t.zero_()
+    graph.replay(); torch.cuda.synchronize()
+    for a, b in zip(want, (Y,) + grads):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
