@@ -55,6 +55,7 @@ constexpr int kSmemBudget = 224 * 1024;              // operand stages plus the 
 constexpr int kStagingPerWarp = 8192;                // two 4 KiB buffers of 32 rows x 128 bytes
 constexpr int EPI_STORE_F32 = 5;                     // like EPI_STORE with fp32 output
 constexpr unsigned long long kWaitNs = 2000000000ull;
+constexpr int kWideMinK = 2048;                      // contraction length from which a CTA pair takes 256 x 512 tiles
 
 // bn = rows of B one CTA loads per k-block (BN / CTAS)
 __host__ __device__ constexpr int stage_bytes(int bn) { return kABytes + bn * BK * 2; }
@@ -273,6 +274,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmC2, const TcParams p) {
   constexpr int BNL = BN / CTAS;                    // rows of B this CTA loads
+  constexpr int kMmaN = BN > 256 ? 256 : BN;        // columns of one MMA; a 512-wide tile takes two per K step
+  constexpr int kBHalf = kMmaN / CTAS;              // rows of B this CTA contributes to one MMA
+  constexpr bool kOneAcc = BN > 256;                // the tile fills tensor memory: one accumulator, no double buffering
+  static_assert(BN <= 256 || CTAS == 2, "512-wide tiles are for CTA pairs");
   constexpr int TM = BM * CTAS;                     // rows of the tile the CTA (pair) works on
   constexpr bool kXchg = EPI == EPI_SOFTMAX && BN >= 128;            // the softmax epilogue's exchange area replaces a stage
   constexpr int kStaging = staging_bytes(BN, EPI);
@@ -329,7 +334,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int b = tile / (p.tiles_m * p.tiles_n);
         const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
         const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
-        const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
+        // B columns of this CTA: per 256-wide MMA the pair's two halves of kBHalf columns each, side by side
+        const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * kBHalf;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
           const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
@@ -349,9 +355,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (p.b_mn) {
 #pragma unroll
-              for (int j = 0; j < BNL / 64; ++j) tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, bc);
+              for (int j = 0; j < BNL / 64; ++j)
+                tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + (64 * j / kBHalf) * kMmaN + 64 * j % kBHalf, k0, bc);
             } else {
-              tma_load_3d_pair(sb, &tmB, bar, k0, n0, bc);
+#pragma unroll
+              for (int j = 0; j < BNL / kBHalf; ++j) tma_load_3d_pair(sb + j * (kBHalf * 128), &tmB, bar, k0, n0 + j * kMmaN, bc);
             }
           } else {
             const uint32_t bar = full0 + 8 * stage;
@@ -377,14 +385,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ MMA issuer (the leader's, in a pair)
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+                             ((uint32_t)(kMmaN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
       // K-major: 8-row groups 1024 B apart, 32 B per K step inside the swizzle atom.
       // MN-major: 64-wide blocks BK*128 B apart (LBO), 8-row K groups 1024 B apart (SBO), 2 groups per K step.
       const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
       const uint32_t a_step = p.a_mn ? 2048 : 32, b_step = p.b_mn ? 2048 : 32;
       int stage = 0; uint32_t phase = 0; int it = 0;
       for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step, ++it) {
-        const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
+        const int buf = kOneAcc ? 0 : it & 1; const uint32_t use = (uint32_t)(kOneAcc ? it : it >> 1);
         if (!mbar_wait(tempty0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.status, 2)) { gave_up = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
@@ -398,6 +406,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint64_t bd = make_desc(sb + kk * b_step, b_lbo, 1024);
             if constexpr (CTAS == 2) tc_mma_pair(d_tmem, ad, bd, idesc, (kb | kk) != 0);
             else tc_mma(d_tmem, ad, bd, idesc, (kb | kk) != 0);
+            if constexpr (kOneAcc) {                 // the tile's second 256 columns: same A, the next kBHalf rows of B
+              const uint64_t bd2 = make_desc(sb + kBHalf * 128 + kk * b_step, b_lbo, 1024);
+              tc_mma_pair(d_tmem + kMmaN, ad, bd2, idesc, (kb | kk) != 0);
+            }
           }
           // the stage is free (in both CTAs) once these MMAs have read it
           if constexpr (CTAS == 2) tc_commit_pair(empty0 + 8 * stage); else tc_commit(empty0 + 8 * stage);
@@ -419,7 +431,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int b = tile / (p.tiles_m * p.tiles_n);
         const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
         const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
-      const int buf = it & 1; const uint32_t use = (uint32_t)(it >> 1);
+      const int buf = kOneAcc ? 0 : it & 1; const uint32_t use = (uint32_t)(kOneAcc ? it : it >> 1);
       const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
       tc_fence_after();
@@ -686,7 +698,10 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
 
 // 256 columns per tile when the tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
 // streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
-int pick_bn(const TcGemmArgs& g) { return (g.N > 128 && g.M > BM) ? 256 : (g.N > 64 ? 128 : 64); }
+int pick_bn(const TcGemmArgs& g) {
+  if (g.M > BM && g.N >= 512 && g.K >= kWideMinK && g.epi == EPI_STORE) return 512;
+  return (g.N > 128 && g.M > BM) ? 256 : (g.N > 64 ? 128 : 64);
+}
 // Two CTAs per tile when a tile of 256 rows is not mostly padding and the pair's B halves are whole 64-wide blocks.
 int pick_ctas(const TcGemmArgs& g, int bn) { return (bn >= 128 && g.M > BM) ? 2 : 1; }
 
@@ -730,6 +745,9 @@ cudaError_t launch_bn(int bn, int ctas, const CUtensorMap& ta, const CUtensorMap
                       const TcParams& p, cudaStream_t st) {
   {
     if (ctas == 2) {
+      if constexpr (EPI == EPI_STORE || EPI == EPI_STORE_F32) {
+        if (bn == 512) return launch_one<512, EPI, 2>(ta, tb, tc, tc2, p, st);
+      }
       if (bn == 256) return launch_one<256, EPI, 2>(ta, tb, tc, tc2, p, st);
       return launch_one<128, EPI, 2>(ta, tb, tc, tc2, p, st);
     }
@@ -766,7 +784,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, kext, ob, g.lda, g.batch_a, 64, BK)
                                 : make_map(&ta, g.A, kext, g.M, ob, g.lda, g.batch_a, BK, BM);
   const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, kext, ob, g.ldb, g.batch_b, 64, BK)
-                                : make_map(&tb, g.B, kext, g.N, ob, g.ldb, g.batch_b, BK, bnl);
+                                : make_map(&tb, g.B, kext, g.N, ob, g.ldb, g.batch_b, BK, bnl > 128 ? 128 : bnl);
   if (!oka || !okb) return cudaErrorInvalidValue;
   // outputs leave through TMA stores of chunks of 32 rows x 128 bytes (64 bf16 or 32 fp32 columns)
   CUtensorMap tc = ta, tc2 = ta;
