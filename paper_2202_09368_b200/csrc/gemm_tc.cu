@@ -32,6 +32,12 @@
 // 128 rows); tcgen05.commit with a two-CTA multicast releases the stage and publishes the
 // accumulator in both.  Each CTA's epilogue warps drain their own rows and report to the
 // leader's barrier.  Loads never use cluster multicast.
+// A pair takes 256 x 512 tiles (BN = 512) when the contraction is long and the epilogue only converts and
+// stores (GEMM-2, dX_in): two MMAs per K step share the A operand, a k-block costs each SM 48 KiB for twice
+// the accumulators (a quarter less fill per flop, which under a power cap is what the clocks follow), and
+// the one accumulator fills tensor memory, so the epilogue is not overlapped: 4 to 8 store chunks per warp
+// against a main loop of at least 256 MMAs.  The epilogues that evaluate GeLU or GeLU' are bound by
+// their arithmetic and stay on 256-column tiles, where the next tile's main loop hides them.
 //
 // Every wait on an mbarrier is bounded: after about two seconds the kernel records
 // EC_ERR_TIMEOUT in the status word, all roles leave their loops and the CTA exits in order.
@@ -65,7 +71,7 @@ __host__ __device__ constexpr int staging_bytes(int bn_tile, int epi) { return (
 __host__ __device__ constexpr int num_stages(int bn, int staging) {
   return (kSmemBudget - staging) / stage_bytes(bn) > 8 ? 8 : (kSmemBudget - staging) / stage_bytes(bn);
 }
-// Two accumulators of BN columns (a power of two for BN = 64, 128, 256).  A CTA pair takes all 512
+// Two accumulators of BN columns (a power of two for BN = 64, 128, 256), or one of 512.  A CTA pair takes all 512
 // columns, so both CTAs are certain to get base address 0: one tcgen05.mma writes the same
 // tensor-memory address in both.
 __host__ __device__ constexpr int tmem_cols(int bn, int ctas) { return ctas == 2 ? 512 : (2 * bn < 32 ? 32 : 2 * bn); }
@@ -696,7 +702,8 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 256 columns per tile when the tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
+// 512 columns per tile for a CTA pair on a long contraction with a plain store; else 256 columns when the
+// tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
 // streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
 int pick_bn(const TcGemmArgs& g) {
   if (g.M > BM && g.N >= 512 && g.K >= kWideMinK && g.epi == EPI_STORE) return 512;
