@@ -113,7 +113,7 @@ def workload_desc(name, groups=1):
 # of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.2 MB at 4 experts of
 # the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
 # moves E/4 times as much.  None for shapes that were not captured.
-GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 635.2e6 / 4, "cfg4e4": 635.2e6 / 4}
+GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 625.2e6 / 4, "cfg4e4": 625.2e6 / 4}
 
 
 def gemm_traffic(workload, E):

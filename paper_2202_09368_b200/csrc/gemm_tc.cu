@@ -705,8 +705,14 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
 // 512 columns per tile for a CTA pair on a long contraction with a plain store; else 256 columns when the
 // tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
 // streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
-int pick_bn(const TcGemmArgs& g) {
-  if (g.M > BM && g.N >= 512 && g.K >= kWideMinK && g.epi == EPI_STORE) return 512;
+int pick_bn(const TcGemmArgs& g, int pairs) {
+  if (g.M > BM && g.N >= 512 && g.K >= kWideMinK && g.epi == EPI_STORE) {
+    // waves of tiles over the CTA pairs, a 512-column tile counted as 1.92 of a 256-column one (its saving in
+    // fill less its epilogue in the open): padding of N to 512 and a thinner last wave can cost more than that
+    const int64_t rows = (int64_t)((g.M + 2 * BM - 1) / (2 * BM)) * g.batches;
+    const int64_t narrow = (rows * ((g.N + 255) / 256) + pairs - 1) / pairs, wide = (rows * ((g.N + 511) / 512) + pairs - 1) / pairs;
+    if (wide * 192 <= narrow * 100) return 512;
+  }
   return (g.N > 128 && g.M > BM) ? 256 : (g.N > 64 ? 128 : 64);
 }
 // Two CTAs per tile when a tile of 256 rows is not mostly padding and the pair's B halves are whole 64-wide blocks.
@@ -780,7 +786,10 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
 }
 
 cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
-  const int bn = pick_bn(g);
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int bn = pick_bn(g, sms / 2);
   const int ctas = pick_ctas(g, bn);
   const int bnl = bn / ctas;                         // rows of B one CTA loads
   CUtensorMap ta, tb;

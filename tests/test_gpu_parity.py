@@ -39,8 +39,9 @@ def test_fp32_tanh_gelu():
     (2048, 256, 512, 32, 2.0),
     (384, 64, 128, 3, 1.0),        # E not a multiple of 8
     (1024, 192, 448, 64, 0.5),     # k = 8
-    (608, 520, 2072, 2, 1.0),      # k = 304, long contraction over d': 512-column tiles with tails in M, N and K
-    (1024, 1024, 2048, 2, 1.0),    # k = 512: whole 256 x 512 tiles
+    (3040, 1000, 2072, 10, 1.0),   # k = 304, long contraction over d', 20 tile rows: GEMM-2 and dX_in take 512-column
+                                   # tiles (one wave instead of two of 256-column ones), with tails in M, N and K
+    (5120, 1024, 2048, 10, 1.0),   # k = 512: whole 256 x 512 tiles
 ])
 def test_bf16_forward_backward(n, d, dff, E, c):
     li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=0)
