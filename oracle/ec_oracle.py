@@ -128,8 +128,44 @@ def expert_ffn_backward(dX_e_i, X_in_i, Z_i, H_i, W1_i, W2_i, gelu_variant: str 
     return dW1, dW2, dX_in, dH, dZ
 
 
-def route(X, Wg, c: float, S_override=None, groups: int = 1):
+def capped_assignment(S, k: int, b: int, lam: float = 1e-3, iters: int = 100):
+    """Section 3.3 (expert choice with at most b experts per token): the matrix A [e, n] of
+
+        max <S^T, A> + lam * H(A)   s.t.  every row sums to k, every column sums to at most b, 0 <= A <= 1,
+
+    by Dykstra's algorithm with I-projections (Kullback-Leibler projections): starting from exp(S^T / lam), the
+    maximiser without constraints up to a constant factor, the iterate is projected in turn onto the three
+    sets, each projection applied to the iterate times that set's correction factor, which then becomes
+    (what was projected) / (its projection).  One iteration is one round over the three sets in the order
+    the programme lists them.  The I-projections are: rows = k, rescale each row; columns <= b, rescale the
+    columns whose sum exceeds b; entries <= 1, clip.  (The row set is affine: its correction factor is
+    constant along a row and cancels in the rescaling, so none is kept.)  Everything is multiplicative, so
+    the iteration runs on L = log A, where exp(S / lam) neither overflows nor underflows.
+    Returns A after `iters` iterations; entries lie in [0, 1], rows sum to at most k, columns to at most b."""
+    from scipy.special import logsumexp
+    S = np.asarray(S, F64)
+    n, e = S.shape
+    L = S.T / lam                                          # [e, n], log of the starting point
+    q_col = np.zeros(n)                                    # log correction factor of the column set (one per column)
+    q_box = np.zeros((e, n))                               # log correction factor of the box set
+    for _ in range(iters):
+        L = L + (math.log(k) - logsumexp(L, axis=1))[:, None]          # rows sum to k
+        B = L + q_col[None, :]
+        m = np.minimum(0.0, math.log(b) - logsumexp(B, axis=0))        # columns above b are scaled down to b
+        L = B + m[None, :]
+        q_col = -m
+        B = L + q_box
+        L = np.minimum(B, 0.0)                                         # entries above 1 are clipped
+        q_box = B - L
+    return np.exp(L)
+
+
+def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3,
+          cap_iters: int = 100):
     """Eq. 1-2: S, G, I and the token->slot inverse index.
+
+    cap_b > 0 (Section 3.3): the indices are TopK(A, k) of the capped assignment A instead of TopK(S^T, k);
+    the gate weights stay G[i, j] = S[I[i, j], i].  The result then also holds A as [n, e].
 
     groups > 1 (the paper's Limitations section: route several groups of tokens independently):
     X holds `groups` blocks of n rows; Eq. 1-2 are applied to each block on its own with k = n*c/e,
@@ -142,6 +178,13 @@ def route(X, Wg, c: float, S_override=None, groups: int = 1):
     n = N // groups
     k = capacity(n, c, e)
     S = gate(X, Wg) if S_override is None else np.asarray(S_override, F64)
+    if cap_b:
+        A = np.concatenate([capped_assignment(S[g * n:(g + 1) * n], k, cap_b, cap_lambda, cap_iters).T
+                            for g in range(groups)])
+        I = np.concatenate([topk(A[g * n:(g + 1) * n], k)[1] + g * n for g in range(groups)], axis=1)
+        G = np.stack([S[I[i], i] for i in range(e)])
+        row_ptr, slots = inverse_index(I, N)
+        return dict(k=k * groups, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots, A=A)
     parts = [topk(S[g * n:(g + 1) * n], k) for g in range(groups)]
     G = np.concatenate([p[0] for p in parts], axis=1)
     I = np.concatenate([p[1] + g * n for g, p in enumerate(parts)], axis=1)
