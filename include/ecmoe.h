@@ -67,6 +67,10 @@ typedef struct {
   double c;        /* capacity factor (Eq. 1)                                         */
   int32_t dtype;   /* ec_dtype                                                        */
   int32_t gelu;    /* ec_gelu                                                         */
+  /* Section 3.3, expert choice with at most cap_b experts per token; cap_b = 0 switches it off. */
+  int32_t cap_b;     /* b: bound on the column sums of A; needs E*k <= n*b                      */
+  int32_t cap_iters; /* rounds of Dykstra's algorithm (the paper: at most 100), >= 1            */
+  double cap_lambda; /* weight of the entropy term (the paper: 0.001), > 0                      */
 } ec_config;
 
 /* Views into the forward->backward blob (device pointers), for inspection and tests. */
@@ -112,6 +116,23 @@ ec_status ec_saved_view(const ec_config* cfg, void* saved, ec_saved_ptrs* out);
 ec_status ec_route(const ec_config* cfg, const void* X, const void* Wg, float* S, int32_t* I,
                    float* G, int32_t* row_ptr, int32_t* slots, void* ws, size_t ws_bytes,
                    void* cuda_stream);
+
+/*
+ * Section 3.3 on its own: the assignment A of
+ *     max <S^T, A> + cap_lambda * H(A)   s.t.  rows sum to k, columns sum to at most cap_b, 0 <= A <= 1
+ * after cap_iters rounds of Dykstra's algorithm with Kullback-Leibler projections (one round: rows, then
+ * columns, then the box, each applied to the iterate times that set's correction factor), started from
+ * exp(S^T / cap_lambda), computed on log A in fp32.  S [n, E] in, A [n, E] out (token-major like S: A[t, i] is
+ * the section's A[i, t]), entries in [0, 1]; routing groups are solved independently.  With cfg->cap_b > 0
+ * ec_route, ec_route_static and ec_moe_forward run this after the gate and take I = TopK(A, k) (same order and
+ * tie rule as Eq. 2) with G[i, j] = S[I[i, j], i]; everything downstream, the backward pass included, is
+ * unchanged (I is a constant there).  This entry point exists to inspect A; it needs cfg->cap_b > 0
+ * (EC_ERR_INVALID_ARG otherwise) and the workspace of ec_workspace_bytes.  At cap_lambda = 0.001 the iteration
+ * advances about log(k / current row sum) per round in log A, so whether the stated 100 rounds reach rows that
+ * sum to k depends on how the scores are spread; cap_iters is the caller's to raise.
+ */
+ec_status ec_capped_assignment(const ec_config* cfg, const float* S, float* A, void* ws, size_t ws_bytes,
+                               void* cuda_stream);
 
 /*
  * The shuffle of Eq. 3 on its own: X_in[i, j, :] = X[I[i, j], :] (X_in = P . X with P = Onehot(I)),

@@ -23,13 +23,14 @@ EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
            "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
-           "ec_forward_only_workspace_bytes"]
+           "ec_forward_only_workspace_bytes", "ec_capped_assignment"]
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class ec_config(C.Structure):
     _fields_ = [("n", C.c_int64), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32),
-                ("groups", C.c_int32), ("c", C.c_double), ("dtype", C.c_int32), ("gelu", C.c_int32)]
+                ("groups", C.c_int32), ("c", C.c_double), ("dtype", C.c_int32), ("gelu", C.c_int32),
+                ("cap_b", C.c_int32), ("cap_iters", C.c_int32), ("cap_lambda", C.c_double)]
 
 
 class ec_saved_ptrs(C.Structure):
@@ -62,6 +63,7 @@ def lib():
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
+        L.ec_capped_assignment.restype = C.c_int; L.ec_capped_assignment.argtypes = [P, V, V, V, C.c_size_t, V]
         L.ec_shuffle.restype = C.c_int; L.ec_shuffle.argtypes = [P, V, V, V, V]
         L.ec_unshuffle.restype = C.c_int; L.ec_unshuffle.argtypes = [P, V, V, V, V, V, V]
         L.ec_moe_forward.restype = C.c_int
@@ -83,10 +85,12 @@ def status_string(code: int) -> str:
     return lib().ec_status_string(code).decode()
 
 
-def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=1) -> ec_config:
+def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=1, cap_b=0, cap_iters=100,
+                cap_lambda=1e-3) -> ec_config:
+    """cap_b > 0: at most cap_b experts per token (Section 3.3) with the paper's solver settings as defaults."""
     dt = {torch.float32: EC_F32, torch.bfloat16: EC_BF16}[dtype]
     return ec_config(int(n), int(d_model), int(d_ff), int(E), int(groups), float(c), dt,
-                     {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu])
+                     {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu], int(cap_b), int(cap_iters), float(cap_lambda))
 
 
 def ec_capacity(cfg: ec_config) -> int:
@@ -170,6 +174,16 @@ def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
     _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
                           _ptr(out.row_ptr), _ptr(out.slots), _ptr(ws), ws.numel(), _stream()), "ec_route")
     return out
+
+
+def ec_capped_assignment(cfg, S, ws=None, A=None):
+    """Section 3.3: A [n, E] after cfg.cap_iters rounds of the solver, from the gate scores S [n, E]."""
+    if A is None:
+        A = torch.empty_like(S)
+    ws = alloc_workspace(cfg, S.device) if ws is None else ws
+    _check(lib().ec_capped_assignment(C.byref(cfg), _ptr(S), _ptr(A), _ptr(ws), ws.numel(), _stream()),
+           "ec_capped_assignment")
+    return A
 
 
 def ec_shuffle(cfg, X, I, X_in=None):

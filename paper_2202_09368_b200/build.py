@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libecmoe.so")
 OBJ = os.path.join(HERE, "_build")
-SOURCES = ["api.cu", "routing.cu", "gemm_simt.cu", "gemm_tc.cu"]
+SOURCES = ["api.cu", "routing.cu", "capped.cu", "gemm_simt.cu", "gemm_tc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
          "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DECMOE_BUILD"]

@@ -18,7 +18,8 @@ inline size_t esize(int dtype) { return dtype == EC_F32 ? 4 : 2; }
 
 // n: all tokens of the call (groups * tokens per group), k: slots per expert (groups * k per group),
 // slots = E * k; ng, kg: the per-group values Eq. 1 is about.
-struct Dims { int64_t n, k, slots, ng, kg; int d, dff, E, groups; int dtype, gelu; size_t eb; };
+struct Dims { int64_t n, k, slots, ng, kg; int d, dff, E, groups; int dtype, gelu; size_t eb;
+              int cap_b, cap_iters; double cap_lambda; };
 
 ec_status check_cfg(const ec_config* c, Dims* D) {
   if (!c) return EC_ERR_INVALID_ARG;
@@ -32,9 +33,15 @@ ec_status check_cfg(const ec_config* c, Dims* D) {
   const int64_t k = ec_capacity(c);
   if (k < 1) return EC_ERR_INVALID_ARG;
   if ((int64_t)c->E * k * c->groups >= ((int64_t)1 << 31)) return EC_ERR_UNSUPPORTED;
+  if (c->cap_b < 0) return EC_ERR_INVALID_ARG;
+  if (c->cap_b > 0) {
+    if (c->cap_iters < 1 || !(c->cap_lambda > 0.0)) return EC_ERR_INVALID_ARG;
+    if ((int64_t)c->E * k > c->n * (int64_t)c->cap_b) return EC_ERR_INVALID_ARG;     // E*k slots cannot fit under the cap
+  }
   if (D) { D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
            D->slots = (int64_t)c->E * D->k; D->d = c->d_model; D->dff = c->d_ff;
-           D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb; }
+           D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb;
+           D->cap_b = c->cap_b; D->cap_iters = c->cap_iters; D->cap_lambda = c->cap_lambda; }
   return EC_OK;
 }
 
@@ -66,7 +73,7 @@ int dwg_splits(const Dims& D) {
   return (int)(p < 1 ? 1 : (p > 32 ? 32 : p));
 }
 
-struct WsLayout { size_t status, topk, inverse, fwd_end, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
+struct WsLayout { size_t status, topk, inverse, cap_A, capped, fwd_end, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
 WsLayout ws_layout(const Dims& D) {
   WsLayout L; size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
@@ -74,6 +81,8 @@ WsLayout ws_layout(const Dims& D) {
   const size_t base = o;
   L.topk = take(topk_scratch_bytes(D.ng, D.E, D.kg, D.groups));
   L.inverse = take(inverse_scratch_bytes(D.n));
+  L.cap_A = take(D.cap_b ? (size_t)D.n * D.E * 4 : 0);
+  L.capped = take(D.cap_b ? capped_scratch_bytes(D.n, D.E, D.groups) : 0);
   const size_t fwd_end = o;
   L.fwd_end = fwd_end;
   o = base;                                   // the backward pass reuses the same region
@@ -166,7 +175,16 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
   }
   if (!done) EC_CUDA(launch_gate_softmax_simt(D.dtype, X, Wg, S, D.n, D.d, D.E, st));
   prof_mark("gate_softmax", st);
-  EC_CUDA(launch_topk(S, D.ng, D.E, D.kg, D.groups, I, G, ws + W.topk, st));
+  const float* keys = S;
+  if (D.cap_b) {                                    // Section 3.3: TopK(A, k) instead of TopK(S^T, k)
+    float* A = (float*)(ws + W.cap_A);
+    EC_CUDA(launch_capped_assignment(S, D.ng, D.E, D.kg, D.groups, D.cap_b, D.cap_iters, (float)D.cap_lambda, A,
+                                     ws + W.capped, st));
+    prof_mark("capped_assignment", st);
+    keys = A;
+  }
+  EC_CUDA(launch_topk(keys, D.ng, D.E, D.kg, D.groups, I, G, ws + W.topk, st));
+  if (D.cap_b) EC_CUDA(launch_gather_gate(S, I, G, D.slots, D.k, D.E, st));      // the gate weights stay S at I
   prof_mark("topk", st);
   EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
   prof_mark("inverse_index", st);
@@ -198,7 +216,7 @@ ec_status static_scratch(void** out) {
 
 // Bytes of scratch the routing stages alone use (the status word, the selection state and the
 // inverse-index cursor); the backward buffers that share the workspace are not part of it.
-size_t route_scratch_bytes(const Dims& D, const WsLayout& W) { return W.inverse + up(inverse_scratch_bytes(D.n)); }
+size_t route_scratch_bytes(const Dims& D, const WsLayout& W) { (void)D; return W.fwd_end; }
 
 }  // namespace
 
@@ -250,6 +268,21 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   prof_begin(st, 0);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
+}
+
+ec_status ec_capped_assignment(const ec_config* c, const float* S, float* A, void* ws, size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!D.cap_b) return EC_ERR_INVALID_ARG;
+  if (!S || !A || !ws || misaligned(S, 16) || misaligned(A, 16) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D);
+  if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  prof_begin(st, 0);
+  EC_CUDA(launch_capped_assignment(S, D.ng, D.E, D.kg, D.groups, D.cap_b, D.cap_iters, (float)D.cap_lambda, A,
+                                   (char*)ws + W.capped, st));
+  prof_mark("capped_assignment", st);
+  return EC_OK;
 }
 
 ec_status ec_shuffle(const ec_config* c, const void* X, const int32_t* I, void* X_in, void* stream) {

@@ -58,6 +58,16 @@ cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* r
 cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems,
                                    cudaStream_t st);
 
+// ---- capped expert choice, Section 3.3 (capped.cu) ---------------------------------------------
+// A [n, E] (token-major, n = groups * ng): the assignment after `iters` rounds of Dykstra's algorithm with
+// Kullback-Leibler projections, per routing group; entries in [0, 1].  E <= 256.
+size_t capped_scratch_bytes(int64_t n, int E, int groups);
+cudaError_t launch_capped_assignment(const float* S, int64_t ng, int E, int64_t kg, int groups, int b, int iters,
+                                     float lambda, float* A, void* scratch, cudaStream_t st);
+// G[i, j] = S[I[i, j], i] for I, G of shape [E, k]
+cudaError_t launch_gather_gate(const float* S, const int32_t* I, float* G, int64_t slots_total, int64_t k, int E,
+                               cudaStream_t st);
+
 // ---- plain FMA GEMM (gemm_simt.cu) -------------------------------------------------------------
 enum Epilogue { EPI_STORE = 0, EPI_GELU = 1, EPI_GELU_GRAD = 2, EPI_ADD_SLOTS = 3 };
 

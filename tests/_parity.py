@@ -47,13 +47,25 @@ def to_np(t):
     return t.detach().float().cpu().numpy().astype(np.float64) if t.is_floating_point() else t.cpu().numpy()
 
 
+CAP_ATOL = 2e-3      # on entries of A in [0, 1]: fp32 rounding of log A (|log A| up to 1/lambda) carried through the rounds
+
+
 def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
-    """Step (ii): bit-exact routing given the GPU's own S."""
+    """Step (ii): bit-exact routing given the GPU's own S.  With a cap (Section 3.3) the GPU's A is compared with
+    the oracle's by tolerance and the indices must be the oracle's TopK of the GPU's own A, the gate weights S at them."""
     k, n, g = B.ec_capacity(cfg), cfg.n, cfg.groups
     S32 = S_gpu.cpu().numpy()                      # float32 bits, compared as such
-    parts = [O.topk(S32[r * n:(r + 1) * n], k) for r in range(g)]          # every routing group on its own
-    G_ref = np.concatenate([p[0] for p in parts], axis=1)
+    keys = S32
+    if cfg.cap_b:
+        A_gpu = B.ec_capped_assignment(cfg, S_gpu.contiguous()).cpu().numpy()
+        A_ref = np.concatenate([O.capped_assignment(S32[r * n:(r + 1) * n], k, cfg.cap_b, cfg.cap_lambda, cfg.cap_iters).T
+                                for r in range(g)])
+        err = np.abs(A_gpu - A_ref).max()
+        assert A_gpu.min() >= 0 and A_gpu.max() <= 1 and err <= CAP_ATOL, f"A differs by {err}"
+        keys = A_gpu
+    parts = [O.topk(keys[r * n:(r + 1) * n], k) for r in range(g)]         # every routing group on its own
     I_ref = np.concatenate([p[1] + r * n for r, p in enumerate(parts)], axis=1)
+    G_ref = np.stack([S32[I_ref[i], i] for i in range(cfg.E)])             # Eq. 2: G[i, j] = S[I[i, j], i]
     I_np = I_gpu.cpu().numpy()
     assert np.array_equal(I_np, I_ref), f"I differs in {(I_np != I_ref).sum()} of {I_ref.size} slots"
     assert np.array_equal(G_gpu.cpu().numpy().view(np.uint32), G_ref.view(np.uint32))
@@ -63,11 +75,11 @@ def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
     return I_ref
 
 
-def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1):
+def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1, **cap):
     """Runs forward (+ backward) on the GPU and checks every tensor against the oracle.
     n is the number of tokens per routing group; li holds groups * n rows."""
     tol = TOL[dtype]
-    cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups)
+    cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups, **cap)
     dev = "cuda"
     X, Wg, W1, W2 = (t.to(dev) for t in (li.X, li.Wg, li.W1, li.W2))
     ws = B.alloc_workspace(cfg)

@@ -9,6 +9,8 @@ Routing and the index lists are compared bit for bit with the oracle evaluated o
 S; the shuffle is a copy and must be exact; the unshuffle is compared with the fp64 sum of
 Eq. 4 within the final bf16 rounding.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -115,3 +117,54 @@ def test_routing_groups_with_ties_on_the_multi_kernel_path():
     cfg = B.make_config(n, d, 16, E, 2.0, torch.float32, groups=groups)
     r = B.ec_route(cfg, X.cuda(), Wg.cuda())
     check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+@pytest.mark.parametrize("n,E,c,b,iters,lam,groups", [
+    (512, 8, 2.0, 2, 100, 1e-3, 1),          # the paper's settings: lambda = 0.001, 100 rounds
+    (1000, 12, 1.5, 2, 40, 1e-3, 1),         # E not a multiple of 32, ragged n
+    (2048, 64, 2.0, 3, 100, 1e-3, 1),
+    (4096, 256, 2.0, 4, 25, 1e-3, 1),        # eight experts per lane
+    (300, 40, 2.0, 3, 300, 5e-3, 3),         # three groups, solved independently; close to converged
+    (16384, 64, 2.0, 2, 100, 1e-3, 1),       # the 8B/64E layer's routing shape
+])
+def test_capped_routing(n, E, c, b, iters, lam, groups):
+    """Section 3.3: A against the oracle's iterate, I = TopK(A, k) bit for bit on the GPU's own A, G = S at I."""
+    d = 64
+    li = IN.make_layer_inputs(groups * n, d, 8, E, BF16, seed=11, with_grad=False)
+    cfg = B.make_config(n, d, 8, E, c, BF16, groups=groups, cap_b=b, cap_iters=iters, cap_lambda=lam)
+    r = B.ec_route(cfg, li.X.cuda(), li.Wg.cuda())
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+    plain = B.ec_route(B.make_config(n, d, 8, E, c, BF16, groups=groups), li.X.cuda(), li.Wg.cuda())
+    assert torch.equal(plain.S, r.S)
+
+
+def test_capped_routing_converged_moves_tokens_under_the_cap():
+    """Run to convergence, the solver leaves only the few tokens over the cap whose entries of A stay fractional
+    (the solution is near-integer, not integer, and TopK rounds it)."""
+    n, d, E, c, b = 1024, 64, 8, 2.0, 3
+    li = IN.make_layer_inputs(n, d, 8, E, BF16, seed=12, with_grad=False)
+    X, Wg = li.X.cuda(), li.Wg.cuda()
+    over = lambda r: int(((r.row_ptr[1:] - r.row_ptr[:-1]) > b).sum())
+    plain = B.ec_route(B.make_config(n, d, 8, E, c, BF16), X, Wg)
+    capped = B.ec_route(B.make_config(n, d, 8, E, c, BF16, cap_b=b, cap_iters=500, cap_lambda=5e-3), X, Wg)
+    assert over(plain) >= 10 and over(capped) <= over(plain) // 3
+    assert int(capped.row_ptr[-1]) == n * 2
+
+
+@pytest.mark.parametrize("dtype,groups", [(torch.float32, 1), (BF16, 2)])
+def test_capped_layer_forward_backward(dtype, groups):
+    """The whole layer with capped routing: everything after the routing is the uncapped path on other indices."""
+    n, d, dff, E, c = 256, 64, 128, 8, 2.0
+    li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=13)
+    run_and_check(n, d, dff, E, c, dtype, li, groups=groups, cap_b=2, cap_iters=60)
+
+
+def test_capped_config_checks():
+    ok = B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2)
+    fwd_bytes = lambda cfg: int(B.lib().ec_forward_only_workspace_bytes(ctypes.byref(cfg)))
+    assert fwd_bytes(ok) >= fwd_bytes(B.make_config(256, 64, 128, 8, 2.0, BF16)) + 3 * 256 * 8 * 4     # A, log A, box factors
+    for bad in (B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=1),                 # E*k = 2n slots cannot fit under b = 1
+                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2, cap_iters=0),
+                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2, cap_lambda=0.0),
+                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=-1)):
+        assert B.ec_workspace_bytes(bad) == 0
