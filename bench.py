@@ -102,15 +102,17 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def workload_desc(name, groups=1):
+def workload_desc(name, groups=1, cap_b=0, cap_iters=100):
     n, d, dff, E, c = WORKLOADS[name]
     how = "one routing group per GPU" if groups == 1 else f"{groups} routing groups of {n // groups} tokens per GPU"
+    if cap_b:
+        how += f", at most {cap_b} experts per token ({cap_iters} solver rounds)"
     return (f"{name}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} fwd+bwd, bf16 storage / fp32 accumulate, "
             f"{how}")
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
-# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 635.2 MB at 4 experts of
+# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 625.2 MB at 4 experts of
 # the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
 # moves E/4 times as much.  None for shapes that were not captured.
 GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 625.2e6 / 4, "cfg4e4": 625.2e6 / 4}
@@ -189,7 +191,7 @@ def run_reference(args):
     out = {"impl": "reference", "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": v, "unit": "tokens/s",
            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / v,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": workload_desc(args.workload, args.groups)},
+           "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters)},
            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -223,7 +225,7 @@ def run_gpu(args):
     n, d, dff, E, c = WORKLOADS[args.workload]
     bf = torch.bfloat16
     assert n % args.groups == 0
-    cfg = B.make_config(n // args.groups, d, dff, E, c, bf, groups=args.groups)
+    cfg = B.make_config(n // args.groups, d, dff, E, c, bf, groups=args.groups, cap_b=args.cap_b, cap_iters=args.cap_iters)
     seed = rank                                                   # each rank routes its own group
     chunk = 1 << 26
     X = IN.normal_tensor((n, d), 1.0, seed, IN.TID_X, bf, dev, chunk)
@@ -347,7 +349,7 @@ def run_gpu(args):
             "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": world * n / (ms_step * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_desc(args.workload, args.groups),
+            "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
                              if args.workload != "small" else "small case, L2 resident",
                        "tensor_cores": bool(B.ec_uses_tensor_cores(cfg)),
@@ -376,10 +378,12 @@ def run_gpu(args):
 ROUTING_GRID = [(n, E) for n in (4096, 16384, 65536, 262144) for E in (8, 32, 128, 256)]
 
 
-def routing_bytes(n, d, E, c, b=2):
-    """Algorithmic bytes each routing stage has to move (reads + writes), per call."""
+def routing_bytes(n, d, E, c, b=2, cap_iters=0):
+    """Algorithmic bytes each routing stage has to move (reads + writes), per call.  The capped solver reads and
+    writes log A and the box factors (fp32) once per round; that state stays in L2 at these sizes."""
     slots = int(n * c)
     return {
+        "capped_assignment": cap_iters * 4 * n * E * 4 + 2 * n * E * 4,
         "gate_softmax": n * d * b + d * E * b + n * E * 4,
         "topk": n * E * 4 + slots * 8,
         "inverse_index": slots * 4 + (n + 1 + slots) * 4,
@@ -409,7 +413,7 @@ def run_routing(args):
     cases = []
     B.ec_profile_enable(True)
     for n, E in grid:
-        cfg = B.make_config(n, d, 8, E, c, bf)
+        cfg = B.make_config(n, d, 8, E, c, bf, cap_b=args.cap_b, cap_iters=args.cap_iters)
         X = IN.normal_tensor((n, d), 1.0, 0, IN.TID_X, bf, dev, 1 << 26)
         Wg = IN.normal_tensor((d, E), 1.0 / math.sqrt(d), 0, IN.TID_WG, bf, dev, 1 << 26)
         ws = B.alloc_workspace(cfg, dev)
@@ -428,7 +432,7 @@ def run_routing(args):
                     if it >= 3:
                         acc.setdefault(k_, []).append(v_)
         assert B.ec_read_status(ws) == B.EC_OK
-        by = routing_bytes(n, d, E, c)
+        by = routing_bytes(n, d, E, c, cap_iters=args.cap_iters if args.cap_b else 0)
         st = {}
         for k_, v_ in acc.items():
             v_.sort()
@@ -438,8 +442,11 @@ def run_routing(args):
                       "frac_nominal": round(by[k_] / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 3)}
         total_us = sum(v["us"] for v in st.values())
         cases.append({"n": n, "E": E, "d": d, "k": int(n * c / E), "stages": st, "chain_us": round(total_us, 2),
-                      "chain_GBps": round(sum(by.values()) / (total_us * 1e-6) / 1e9, 1),
+                      "chain_GBps": round(sum(by[k_] for k_ in st) / (total_us * 1e-6) / 1e9, 1),
                       "tokens_per_s": round(n / (total_us * 1e-6))})
+        if args.cap_b:                                    # what the cap did to the number of experts per token
+            cases[-1]["cap"] = {"b": args.cap_b, "rounds": args.cap_iters, "lambda": 1e-3,
+                                "experts_per_token_hist": torch.bincount(r.row_ptr[1:] - r.row_ptr[:-1]).tolist()}
         del X, Wg, ws, r, X_in, X_e, X_out
     B.ec_profile_enable(False)
     print(json.dumps({"metric": "ec_routing_chain", "unit": "GB/s (algorithmic bytes / device time per stage)",
@@ -520,6 +527,8 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--graph", action="store_true", help="time the step as one captured CUDA graph")
+    ap.add_argument("--cap-b", type=int, default=0, help="at most this many experts per token (Section 3.3); 0 = plain expert choice")
+    ap.add_argument("--cap-iters", type=int, default=100, help="rounds of the capped solver")
     ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")

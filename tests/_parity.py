@@ -61,6 +61,7 @@ def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
         A_ref = np.concatenate([O.capped_assignment(S32[r * n:(r + 1) * n], k, cfg.cap_b, cfg.cap_lambda, cfg.cap_iters).T
                                 for r in range(g)])
         err = np.abs(A_gpu - A_ref).max()
+        print(f"capped assignment: max |A - oracle| = {err:.2e}")
         assert A_gpu.min() >= 0 and A_gpu.max() <= 1 and err <= CAP_ATOL, f"A differs by {err}"
         keys = A_gpu
     parts = [O.topk(keys[r * n:(r + 1) * n], k) for r in range(g)]         # every routing group on its own
