@@ -16,7 +16,9 @@ distribution over experts); TopK breaks ties toward the lower token index and
 lists each expert's tokens by descending score; GeLU is the exact erf form by
 default (tanh form optional); no biases; G is used raw (no renormalisation);
 a token chosen by no expert gets a zero output row; in the backward pass the
-index matrix I is a constant, so the gate is trained through G only.
+index matrix I is a constant, so the gate is trained through G only; the capped variant
+of Section 3.3 is Dykstra's algorithm with Kullback-Leibler projections, one round = rows,
+columns, box, on log A, and replaces only the indices (see capped_assignment).
 
 Every function here is pinned by tests/test_oracle_*.py against closed forms,
 brute force, invariants, library routines and finite differences; nothing in
