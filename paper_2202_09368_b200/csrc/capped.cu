@@ -37,7 +37,7 @@ constexpr int kCapThreads = 1024;
 constexpr int kCapWarps = kCapThreads / 32;
 constexpr int kCapMaxE = 256;
 constexpr int kCapLoads = 4;                         // partials a thread of the row step has in flight 
-constexpr int kCapBatch = 4;                         // tokens of a warp whose loads are in flight together
+constexpr int kCapBatch = 4;                         // tokens of a warp whose loads are in flight together (fewer with many experts per lane)
 constexpr int kCapResident = 8;                      // (tokens per warp) x (experts per lane) the resident form holds:
                                                      // log A and the box factors of that many entries in a lane's registers
 
@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(kCapThreads)
 capped_round_kernel(const float* __restrict__ S, float* __restrict__ L, float* __restrict__ qb, float* __restrict__ qc,
                     float* __restrict__ A, const float2* __restrict__ part_in, float2* __restrict__ part_out,
                     int64_t ng, int E, float inv_lambda, float log_k, float log_b, int phase, int first, int last) {
+  constexpr int kBatch = EPL >= 8 ? 1 : (EPL >= 4 ? 2 : kCapBatch);   // so that a batch fits the 64 registers of a thread
   extern __shared__ float2 cap_smem[];
   float* shift = shift_of(cap_smem, E);
   const int g = blockIdx.y, bpg = gridDim.x, blk = blockIdx.x;
@@ -139,14 +140,14 @@ capped_round_kernel(const float* __restrict__ S, float* __restrict__ L, float* _
   float pm[EPL], ps[EPL];
 #pragma unroll
   for (int j = 0; j < EPL; ++j) { pm[j] = 0.f; ps[j] = 0.f; }
-  // A warp takes its tokens kCapBatch at a time: the loads of a batch are issued together (they do not depend on
+  // A warp takes its tokens kBatch at a time: the loads of a batch are issued together (they do not depend on
   // the row sums, so the first batch's are in flight while the CTA combines the partials), the arithmetic
   // follows token by token in ascending order.
   const int64_t stride = (int64_t)bpg * kCapWarps;
-  float x[kCapBatch][EPL], qbv[kCapBatch][EPL], qcv[kCapBatch];
+  float x[kBatch][EPL], qbv[kBatch][EPL], qcv[kBatch];
   auto load_batch = [&](int64_t tb) {
 #pragma unroll
-    for (int u = 0; u < kCapBatch; ++u) {
+    for (int u = 0; u < kBatch; ++u) {
       const int64_t t = tb + u * stride;
       const int64_t tok = (int64_t)g * ng + t, row = tok * E;
       qcv[u] = 0.f;
@@ -165,7 +166,7 @@ capped_round_kernel(const float* __restrict__ S, float* __restrict__ L, float* _
   if (phase == 1) row_shifts(part_in, g, bpg, E, log_k, shift);       // every thread of the CTA gets here
   while (tb < ng) {
 #pragma unroll
-    for (int u = 0; u < kCapBatch; ++u) {
+    for (int u = 0; u < kBatch; ++u) {
       const int64_t t = tb + u * stride;
       if (t < ng) {                                                    // uniform across the warp
         const int64_t tok = (int64_t)g * ng + t, row = tok * E;
@@ -188,7 +189,7 @@ capped_round_kernel(const float* __restrict__ S, float* __restrict__ L, float* _
         }
       }
     }
-    tb += kCapBatch * stride;
+    tb += kBatch * stride;
     if (tb < ng) load_batch(tb);
   }
   publish_partials<EPL>(pm, ps, cap_smem, E, part_out, g, bpg, blk);
