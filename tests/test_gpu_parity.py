@@ -134,11 +134,13 @@ def test_forward_only_gives_the_same_output_without_a_saved_blob(dtype, n, d, df
     torch.cuda.synchronize()
 
 
-def test_a_step_can_be_captured_in_a_cuda_graph():
-    """Forward and backward only queue work on the caller's stream: a step captured once replays to the same bits."""
+@pytest.mark.parametrize("cap", [{}, {"cap_b": 3, "cap_iters": 30}])
+def test_a_step_can_be_captured_in_a_cuda_graph(cap):
+    """Forward and backward only queue work on the caller's stream: a step captured once replays to the same bits
+    (with the capped routing too, whose solver is a cooperative launch)."""
     n, d, dff, E = 1024, 128, 256, 8
     li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=5)
-    cfg = B.make_config(n, d, dff, E, 2.0, BF16)
+    cfg = B.make_config(n, d, dff, E, 2.0, BF16, **cap)
     X, Wg, W1, W2, dY = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2, li.dX_out))
     ws, saved, Y = B.alloc_workspace(cfg), B.alloc_saved(cfg), torch.empty_like(X)
     grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
