@@ -42,6 +42,7 @@ def test_fp32_tanh_gelu():
     (3040, 1000, 2072, 10, 1.0),   # k = 304, long contraction over d', 20 tile rows: GEMM-2 and dX_in take 512-column
                                    # tiles (one wave instead of two of 256-column ones), with tails in M, N and K
     (5120, 1024, 2048, 10, 1.0),   # k = 512: whole 256 x 512 tiles
+    (8000, 512, 2056, 40, 1.0),    # k = 200, forty experts of one 256 x 512 tile each (d = 512), ragged K
 ])
 def test_bf16_forward_backward(n, d, dff, E, c):
     li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=0)
