@@ -9,8 +9,6 @@ Routing and the index lists are compared bit for bit with the oracle evaluated o
 S; the shuffle is a copy and must be exact; the unshuffle is compared with the fp64 sum of
 Eq. 4 within the final bf16 rounding.
 """
-import ctypes
-
 import numpy as np
 import pytest
 import torch
@@ -159,14 +157,3 @@ def test_capped_layer_forward_backward(dtype, groups):
     n, d, dff, E, c = 256, 64, 128, 8, 2.0
     li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=13)
     run_and_check(n, d, dff, E, c, dtype, li, groups=groups, cap_b=2, cap_iters=60)
-
-
-def test_capped_config_checks():
-    ok = B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2)
-    fwd_bytes = lambda cfg: int(B.lib().ec_forward_only_workspace_bytes(ctypes.byref(cfg)))
-    assert fwd_bytes(ok) >= fwd_bytes(B.make_config(256, 64, 128, 8, 2.0, BF16)) + 3 * 256 * 8 * 4     # A, log A, box factors
-    for bad in (B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=1),                 # E*k = 2n slots cannot fit under b = 1
-                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2, cap_iters=0),
-                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=2, cap_lambda=0.0),
-                B.make_config(256, 64, 128, 8, 2.0, BF16, cap_b=-1)):
-        assert B.ec_workspace_bytes(bad) == 0

@@ -61,3 +61,16 @@ def test_null_pointers_are_rejected_without_a_gpu():
     assert code == B.EC_ERR_INVALID_ARG
     code = L.ec_moe_forward(ctypes.byref(cfg), None, None, None, None, None, None, 0, None, 0, None)
     assert code == B.EC_ERR_INVALID_ARG
+
+
+def test_capped_config_checks():
+    """Section 3.3 options: the scratch grows by A, log A and the box factors; infeasible or malformed settings are refused
+    by the size functions (host arithmetic only)."""
+    ok = B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16, cap_b=2)
+    fwd_bytes = lambda cfg: int(B.lib().ec_forward_only_workspace_bytes(ctypes.byref(cfg)))
+    assert fwd_bytes(ok) >= fwd_bytes(B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16)) + 3 * 256 * 8 * 4     # A, log A, box factors
+    for bad in (B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16, cap_b=1),                 # E*k = 2n slots cannot fit under b = 1
+                B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16, cap_b=2, cap_iters=0),
+                B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16, cap_b=2, cap_lambda=0.0),
+                B.make_config(256, 64, 128, 8, 2.0, torch.bfloat16, cap_b=-1)):
+        assert B.ec_workspace_bytes(bad) == 0
