@@ -18,6 +18,8 @@
 //   - resident: one cooperative launch for all rounds; a warp keeps log A and the factors of its (at most 8 /
 //     experts-per-lane) tokens in registers, the CTAs meet at a grid barrier once per round and only the row
 //     partials go through memory.  Used whenever the tokens fit (up to about 19 k tokens at 64 experts);
+//   - resident in shared memory: the same launch with the state in the CTA's shared memory, for up to about
+//     2.4 M entries per device (16384 tokens x 128 experts, 65536 x 32);
 //   - one launch per round with the state (2 x 4 bytes per entry) in global memory, where it stays in L2 at
 //     the layer sizes.  For everything else.
 // Either way a round costs latency (a barrier or a launch, one round trip for the partials, the reduction
@@ -248,6 +250,75 @@ capped_resident_kernel(const float* __restrict__ S, float* __restrict__ A, float
   }
 }
 
+// The same with the state in shared memory instead of registers, for groups whose tokens do not fit the registers:
+// behind wpart and shift come log A and the box factors of the warp's tokens ([warp][token][2][E]) and the column
+// factors ([warp][token]).  A warp touches only its own part, so no barrier guards it.
+template <int EPL>
+__global__ void __launch_bounds__(kCapThreads)
+capped_resident_smem_kernel(const float* __restrict__ S, float* __restrict__ A, float2* __restrict__ part0,
+                            float2* __restrict__ part1, int64_t ng, int E, float inv_lambda, float log_k, float log_b,
+                            int iters, int tpw) {
+  extern __shared__ float2 cap_smem[];
+  float* shift = shift_of(cap_smem, E);
+  cg::grid_group grid = cg::this_grid();
+  const int g = blockIdx.y, bpg = gridDim.x, blk = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t stride = (int64_t)bpg * kCapWarps, t0 = (int64_t)blk * kCapWarps + warp;
+  float* mine = shift + E + (size_t)warp * tpw * 2 * E;            // this warp's tokens: [token][log A | box factor][E]
+  float* my_qc = shift + E + (size_t)kCapWarps * tpw * 2 * E + warp * tpw;
+  float pm[EPL], ps[EPL];
+#pragma unroll
+  for (int j = 0; j < EPL; ++j) { pm[j] = 0.f; ps[j] = 0.f; }
+  for (int u = 0; u < tpw; ++u) {
+    const int64_t t = t0 + u * stride, row = ((int64_t)g * ng + t) * E;
+    if (t < ng) {                                    // uniform across the warp
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) {
+        const int i = lane + 32 * j;
+        if (i < E) {
+          const float v = S[row + i] * inv_lambda;
+          mine[(2 * u) * E + i] = v; mine[(2 * u + 1) * E + i] = 0.f;
+          lse_add(pm[j], ps[j], v, 1.f);
+        }
+      }
+      if (lane == 0) my_qc[u] = 0.f;
+    }
+  }
+  publish_partials<EPL>(pm, ps, cap_smem, E, part0, g, bpg, blk);
+  for (int it = 0; it < iters; ++it) {
+    grid.sync();                                     // every CTA's partials of the previous pass are in memory
+    row_shifts((it & 1) ? part1 : part0, g, bpg, E, log_k, shift);
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) { pm[j] = 0.f; ps[j] = 0.f; }
+    for (int u = 0; u < tpw; ++u) {
+      if (t0 + u * stride < ng) {                    // uniform across the warp
+        float x[EPL], qb[EPL];
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+          const int i = lane + 32 * j;
+          x[j] = i < E ? mine[(2 * u) * E + i] + shift[i] : -INFINITY;                               // rows sum to k
+          qb[j] = i < E ? mine[(2 * u + 1) * E + i] : 0.f;
+        }
+        float qc = my_qc[u];
+        __syncwarp();                                // every lane has read the column factor before lane 0 rewrites it
+        token_round<EPL>(x, qb, qc, lane, E, log_b);
+        if (lane == 0) my_qc[u] = qc;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+          const int i = lane + 32 * j;
+          if (i < E) { mine[(2 * u) * E + i] = x[j]; mine[(2 * u + 1) * E + i] = qb[j]; ps[j] += __expf(x[j]); }
+        }
+      }
+    }
+    if (it + 1 < iters) publish_partials<EPL>(pm, ps, cap_smem, E, (it & 1) ? part0 : part1, g, bpg, blk);
+  }
+  for (int u = 0; u < tpw; ++u) {
+    const int64_t t = t0 + u * stride, row = ((int64_t)g * ng + t) * E;
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) if (t < ng && lane + 32 * j < E) A[row + lane + 32 * j] = __expf(mine[(2 * u) * E + lane + 32 * j]);
+  }
+}
+
 __global__ void gather_gate_kernel(const float* __restrict__ S, const int32_t* __restrict__ I, float* __restrict__ G,
                                    int64_t slots_total, int64_t k, int E) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < slots_total; s += (int64_t)gridDim.x * blockDim.x)
@@ -293,6 +364,23 @@ cudaError_t launch_resident_tpw(int tpw, ResidentArgs a, dim3 grid, int sms, boo
   return cudaSuccess;
 }
 
+constexpr size_t kCapSmemLimit = 200 * 1024;         // of a CTA's 227 KiB
+template <int EPL>
+cudaError_t launch_resident_smem(ResidentArgs a, int tpw, dim3 grid, int sms, bool* fits, cudaStream_t st) {
+  auto kern = capped_resident_smem_kernel<EPL>;
+  const size_t smem = cap_smem_bytes(a.E) + (size_t)kCapWarps * tpw * (2 * a.E + 1) * 4;
+  *fits = false;
+  if (smem > kCapSmemLimit) return cudaSuccess;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCapSmemLimit) != cudaSuccess) return cudaErrorInvalidValue;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kCapThreads, smem) != cudaSuccess) return cudaErrorInvalidValue;
+  *fits = (int64_t)per_sm * sms >= (int64_t)grid.x * grid.y;
+  if (!*fits) return cudaSuccess;
+  void* args[] = {&a.S, &a.A, &a.part0, &a.part1, &a.ng, &a.E, &a.inv_lambda, &a.log_k, &a.log_b, &a.iters, &tpw};
+  count_launch();
+  return cudaLaunchCooperativeKernel((void*)kern, grid, dim3(kCapThreads), args, smem, st);
+}
+
 }  // namespace
 
 // scratch: L [n, E] | qb [n, E] | qc [n] | two sets of row partials
@@ -328,6 +416,16 @@ cudaError_t launch_capped_assignment(const float* S, int64_t ng, int E, int64_t 
                   : epl == 2 ? launch_resident_tpw<2>((int)tpw, a, grid, sms, &fits, st)
                   : epl == 4 ? launch_resident_tpw<4>((int)tpw, a, grid, sms, &fits, st)
                              : launch_resident_tpw<8>((int)tpw, a, grid, sms, &fits, st);
+    if (e != cudaSuccess) return e;
+    if (fits) return cudaGetLastError();
+  }
+  if (coop && tpw * epl > kCapResident && tpw <= 1024) {             // too many entries for registers: try shared memory
+    ResidentArgs a{S, A, part[0], part[1], ng, E, inv_lambda, log_k, log_b, iters};
+    bool fits = false;
+    cudaError_t e = epl == 1 ? launch_resident_smem<1>(a, (int)tpw, grid, sms, &fits, st)
+                  : epl == 2 ? launch_resident_smem<2>(a, (int)tpw, grid, sms, &fits, st)
+                  : epl == 4 ? launch_resident_smem<4>(a, (int)tpw, grid, sms, &fits, st)
+                             : launch_resident_smem<8>(a, (int)tpw, grid, sms, &fits, st);
     if (e != cudaSuccess) return e;
     if (fits) return cudaGetLastError();
   }
