@@ -124,8 +124,8 @@ def test_routing_groups_with_ties_on_the_multi_kernel_path():
     (4096, 256, 2.0, 4, 25, 1e-3, 1),        # eight experts per lane
     (300, 40, 2.0, 3, 300, 5e-3, 3),         # three groups, solved independently; close to converged
     (16384, 64, 2.0, 2, 100, 1e-3, 1),       # the 8B/64E layer's routing shape
-    (40000, 64, 2.0, 2, 12, 1e-3, 1),        # too many tokens for the register-resident form: one launch per round
-    (9000, 200, 2.0, 3, 7, 1e-3, 2),         # the same form with seven experts per lane and two groups
+    (40000, 64, 2.0, 2, 12, 1e-3, 1),        # too many tokens for the registers: state in shared memory
+    (9000, 200, 2.0, 3, 7, 1e-3, 2),         # too much for shared memory too (seven experts per lane, two groups): one launch per round
 ])
 def test_capped_routing(n, E, c, b, iters, lam, groups):
     """Section 3.3: A against the oracle's iterate, I = TopK(A, k) bit for bit on the GPU's own A, G = S at I."""
