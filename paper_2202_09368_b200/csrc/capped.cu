@@ -63,7 +63,9 @@ __device__ __forceinline__ float* shift_of(float2* smem, int E) { return reinter
 // shift[i] = log k - log(sum over the group's tokens of exp L[:, i]) from the partials the CTAs of group g left.
 // P adjacent lanes share an expert: each combines every P-th CTA's partial in ascending order (loads several at
 // a time, kCapLoads in flight), a butterfly joins them.  Every thread of the CTA calls this.
-__device__ __forceinline__ void row_shifts(const float2* __restrict__ part_in, int g, int bpg, int E, float log_k, float* shift) {
+// The partials were written by other CTAs, in the resident forms by the same launch: they are read from L2
+// (ld.global.cg), never through a read-only or L1 path that could hold the values of two rounds ago.
+__device__ __forceinline__ void row_shifts(const float2* part_in, int g, int bpg, int E, float log_k, float* shift) {
   int P = 32;
   while (P * E > kCapThreads) P >>= 1;               // E <= 256: P >= 4
   const int i = threadIdx.x / P, p0 = threadIdx.x % P;
@@ -74,7 +76,7 @@ __device__ __forceinline__ void row_shifts(const float2* __restrict__ part_in, i
 #pragma unroll
       for (int u = 0; u < kCapLoads; ++u) {
         const int qq = q + u * P;
-        v[u] = qq < bpg ? part_in[((int64_t)g * E + i) * bpg + qq] : make_float2(0.f, 0.f);      // adjacent lanes, adjacent CTAs
+        v[u] = qq < bpg ? __ldcg(part_in + ((int64_t)g * E + i) * bpg + qq) : make_float2(0.f, 0.f);   // adjacent lanes, adjacent CTAs
       }
 #pragma unroll
       for (int u = 0; u < kCapLoads; ++u) lse_add(m, s, v[u].x, v[u].y);
