@@ -21,8 +21,12 @@ of Section 3.3 is Dykstra's algorithm with Kullback-Leibler projections, one rou
 columns, box, on log A, and replaces only the indices (see capped_assignment).
 
 Every function here is pinned by tests/test_oracle_*.py against closed forms,
-brute force, invariants, library routines and finite differences; nothing in
-this file is "parity unpinned".
+brute force, invariants, library routines and finite differences, the `store=`
+hook of forward() / backward() included (tests/test_oracle_store_hook.py: the
+identity hook is bitwise the definition, the names it sees are fixed, and what a
+bf16-rounding hook does to each output is bracketed by the single-rounding error
+of that output and stored under tests/golden/); nothing in this file is
+"parity unpinned".
 """
 from __future__ import annotations
 
@@ -112,7 +116,10 @@ def gelu_grad(z, variant: str = "erf"):
 
 
 def expert_ffn(X_in_i, W1_i, W2_i, gelu_variant: str = "erf", store=_keep):
-    """Eq. 3 for one expert: Z = X_in[i] . W1[i], H = GeLU(Z), X_e[i] = H . W2[i]^T."""
+    """Eq. 3 for one expert: Z = X_in[i] . W1[i], H = GeLU(Z), X_e[i] = H . W2[i]^T.
+
+    `store` (see forward()) is handed every tensor this function produces.  H is GeLU of the product
+    itself, as Eq. 3 writes it, not of what `store` made of Z."""
     Z = X_in_i @ W1_i                                      # [k, d']
     H = store("H", gelu(Z, gelu_variant))
     Z = store("Z", Z)
@@ -124,10 +131,10 @@ def expert_ffn_backward(dX_e_i, X_in_i, Z_i, H_i, W1_i, W2_i, gelu_variant: str 
     """Chain rule through Eq. 3 for one expert; returns dW1[i], dW2[i], dX_in[i], dH, dZ."""
     dH = dX_e_i @ W2_i                                     # [k, d']
     dW2 = store("dW2", dX_e_i.T @ H_i)                     # [d, d']
-    dZ = store("dZ", dH * gelu_grad(Z_i, gelu_variant))
+    dZ = store("dZ", dH * gelu_grad(Z_i, gelu_variant))    # dH is consumed here as computed; it is handed to `store` on return
     dW1 = store("dW1", X_in_i.T @ dZ)                      # [d, d']
     dX_in = store("dX_in", dZ @ W1_i.T)                    # [k, d]
-    return dW1, dW2, dX_in, dH, dZ
+    return dW1, dW2, dX_in, store("dH", dH), dZ
 
 
 def capped_assignment(S, k: int, b: int, lam: float = 1e-3, iters: int = 100):
@@ -195,23 +202,28 @@ def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap
 
 
 def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
-            store=_keep, groups: int = 1):
+            store=_keep, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3, cap_iters: int = 100):
     """Eq. 1-4.  Returns every intermediate.
 
     S_override replaces the gate output (the routing is then taken from it);
     I_override additionally fixes the index matrix (G is read from S at I).
     Both exist so that later stages can be compared on identical routing.
 
-    `store(name, array)` is applied to each tensor at the point where the layer
-    keeps it in memory (Z, H, X_e, X_out).  The default keeps fp64, which is the
-    definition; a test passes a rounding function to measure how far a storage
-    format alone moves the result (the arithmetic floor of a low-precision path).
+    cap_b > 0 routes with the capped assignment of Section 3.3 (see route()).
+
+    `store(name, array)` is handed EVERY named tensor the layer produces after the routing
+    (X_in, Z, H, X_e, X_out here; dX_e, dG, dH, dZ, dW1, dW2, dX_in, dS, dL, dWg, dX in backward()),
+    once, at the point where the definition has finished computing it, and what it returns is
+    what later steps read.  The default returns its argument, which is the definition in fp64.
+    A test may pass a function that rounds the tensors of its choosing to a storage format, to
+    measure how far that format alone moves the result; which tensors those are is the test's
+    business, this file knows nothing of any implementation's storage.
     """
     X = np.asarray(X, F64); Wg = np.asarray(Wg, F64)
     W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
     n, d = X.shape
     e = Wg.shape[1]
-    r = route(X, Wg, c, S_override, groups)
+    r = route(X, Wg, c, S_override, groups, cap_b, cap_lambda, cap_iters)
     k, S = r["k"], r["S"]
     if I_override is not None:
         I = np.asarray(I_override, np.int64)
@@ -219,7 +231,7 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
         row_ptr, slots = inverse_index(I, n)
         r.update(I=I, G=G, row_ptr=row_ptr, slots=slots)
     I, G = r["I"], r["G"]
-    X_in = X[I]                                            # Eq. 3: X_in = P . X,  [e, k, d]
+    X_in = store("X_in", X[I])                             # Eq. 3: X_in = P . X,  [e, k, d]
     per_expert = [expert_ffn(X_in[i], W1[i], W2[i], gelu_variant, store) for i in range(e)]
     Z = np.stack([p[0] for p in per_expert])               # [e, k, d']
     H = np.stack([p[1] for p in per_expert])               # [e, k, d']
@@ -246,7 +258,7 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     k = I.shape[1]
     dY = dX_out[I]                                         # [e, k, d] rows of dX_out seen by each slot
     dX_e = store("dX_e", G[:, :, None] * dY)               # Eq. 4 w.r.t. X_e
-    dG = np.einsum("ijd,ijd->ij", dY, X_e)                 # Eq. 4 w.r.t. G
+    dG = store("dG", np.einsum("ijd,ijd->ij", dY, X_e))    # Eq. 4 w.r.t. G
     per_expert = [expert_ffn_backward(dX_e[i], X_in[i], Z[i], H[i], W1[i], W2[i], gelu_variant, store)
                   for i in range(e)]
     dW1 = np.stack([p[0] for p in per_expert])             # [e, d, d']
@@ -257,6 +269,7 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     dS = np.zeros((n, e), F64)
     for i in range(e):
         dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
+    dS = store("dS", dS)
     dL = store("dL", S * (dS - (dS * S).sum(axis=1, keepdims=True)))   # softmax Jacobian, per token row
     dWg = store("dWg", X.T @ dL)
     dX = dL @ Wg.T

@@ -16,7 +16,7 @@ def layer_onehot(X, Wg, W1, W2, c):
     W1 = np.asarray(W1, np.float64); W2 = np.asarray(W2, np.float64)
     n, d = X.shape
     e = Wg.shape[1]
-    k = int(round(n * c / e))
+    k = int(math.floor(n * c / e + 1e-9))              # Eq. 1, non-integer values floored
     logits = np.einsum("nd,de->ne", X, Wg)
     ex = np.exp(logits - logits.max(axis=1, keepdims=True))
     S = ex / ex.sum(axis=1, keepdims=True)

@@ -14,7 +14,9 @@ are tensor-core operands or bf16 activations by definition of the path), and its
 outputs are heavy-tailed (a token's row scales with its gate weights), so the
 exact fp64 result rounded once to bf16 can sit above 2e-2 by itself.  The test
 therefore also evaluates the oracle with those tensors rounded to bf16 where they
-are stored (the arithmetic floor, CPU only) and accepts max(2e-2, 1.5 x floor).
+are stored (the arithmetic floor, CPU only; tests/test_oracle_store_hook.py pins what
+that floor may be) and accepts max(2e-2, FLOOR_SLACK x floor): the kernels may add a
+tenth of the format's own rounding on top of it, no more.
 """
 import numpy as np
 import torch
@@ -22,7 +24,15 @@ import torch
 from oracle import ec_oracle as O
 from paper_2202_09368_b200 import binding as B
 
+from _storage import BF16_STORED, bf16_store  # noqa: F401  (re-exported to the test modules)
+
 TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}
+FLOOR_SLACK = 1.1
+
+
+def bf16_bound(floor):
+    """Bound on a bf16-path tensor whose storage floor (see the module text) is `floor`."""
+    return max(TOL[torch.bfloat16], FLOOR_SLACK * floor)
 
 
 def rel_err(got, ref):
@@ -31,16 +41,6 @@ def rel_err(got, ref):
     if rms == 0:
         return float(np.max(np.abs(got)))
     return float(np.max(np.abs(got - ref)) / rms)
-
-
-BF16_STORED = {"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2"}
-
-
-def bf16_store(name, x):
-    """Storage rounding of the bf16 path: round-to-nearest-even to bf16 where the layer keeps bf16."""
-    if name not in BF16_STORED:
-        return x
-    return torch.from_numpy(np.ascontiguousarray(x, np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
 
 
 def to_np(t):
@@ -115,7 +115,7 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         if backward:
             fb = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), ff, gelu, store=bf16_store)
             floor.update({k_: rel_err(fb[k_], b[k_]) for k_ in ("dX", "dWg", "dW1", "dW2")})
-        bound = {k_: max(tol, 1.5 * floor.get(k_, 0.0)) for k_ in errs}
+        bound = {k_: bf16_bound(floor.get(k_, 0.0)) for k_ in errs}
         errs["_floor"] = floor
     bad = {k_: (e, bound[k_]) for k_, e in errs.items() if k_ in bound and not e <= bound[k_]}
     assert not bad, f"over tolerance (err, bound): {bad} (all: {errs})"

@@ -16,7 +16,7 @@ from oracle import ec_oracle as O
 from paper_2202_09368_b200 import binding as B
 from paper_2202_09368_b200 import inputs as IN
 
-from _parity import TOL, bf16_store, check_routing, rel_err, run_and_check, to_np
+from _parity import TOL, bf16_bound, bf16_store, check_routing, rel_err, run_and_check, to_np
 
 pytestmark = pytest.mark.gpu
 BF16 = torch.bfloat16
@@ -29,8 +29,7 @@ def test_100m_32e_layer_full_parity():
     print({k: (f"{v:.3e}" if not isinstance(v, dict) else v) for k, v in errs.items()})
 
 
-def _bound(err_floor):
-    return max(TOL[BF16], 1.5 * err_floor)
+_bound = bf16_bound
 
 
 def test_8b_64e_layer_sampled_parity():

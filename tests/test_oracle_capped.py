@@ -126,3 +126,21 @@ def test_groups_are_capped_independently():
         one = O.route(np.zeros((n, 1)), np.zeros((1, e)), c, S_override=S[g * n:(g + 1) * n], cap_b=b, cap_iters=50)
         assert np.array_equal(many["I"][:, g * k:(g + 1) * k], one["I"] + g * n)
         assert np.array_equal(many["A"][g * n:(g + 1) * n], one["A"])
+
+
+def test_forward_with_a_cap_routes_with_the_capped_indices():
+    """oracle.forward(cap_b=...) is route(cap_b=...) followed by the uncapped Eq. 3-4 on those indices."""
+    import torch
+    from paper_2202_09368_b200 import inputs as IN
+    li = IN.make_layer_inputs(96, 16, 24, 4, torch.float32, seed=2)
+    X, Wg, W1, W2 = (t.numpy().astype(np.float64) for t in (li.X, li.Wg, li.W1, li.W2))
+    cap = dict(cap_b=2, cap_lambda=5e-3, cap_iters=200)
+    r = O.route(X, Wg, 2.0, **cap)
+    f = O.forward(X, Wg, W1, W2, 2.0, **cap)
+    plain = O.forward(X, Wg, W1, W2, 2.0)
+    assert np.array_equal(f["I"], r["I"]) and np.array_equal(f["G"], r["G"]) and np.array_equal(f["A"], r["A"])
+    assert not np.array_equal(f["I"], plain["I"])                    # the cap moved some tokens
+    again = O.forward(X, Wg, W1, W2, 2.0, I_override=r["I"])         # same indices through the uncapped path
+    assert np.array_equal(f["X_out"], again["X_out"])
+    per_token = O.experts_per_token(f["row_ptr"])
+    assert per_token.sum() == 96 * 2 and (per_token > 2).sum() < (O.experts_per_token(plain["row_ptr"]) > 2).sum()
