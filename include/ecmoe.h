@@ -32,8 +32,12 @@
  *  - X, Wg, W1, W2, X_out, dX_out and all gradients have the element type
  *    cfg->dtype; S, G and X_e are always fp32 and index outputs are int32.
  *  - Restrictions (EC_ERR_UNSUPPORTED otherwise): d_model and d_ff rows must be a
- *    multiple of 16 bytes long; groups*n < 2^31; 1 <= E <= 256; E*groups*k < 2^31;
- *    1 <= groups <= 65535.
+ *    multiple of 16 bytes long and d_model, d_ff <= 2^22 - 64; groups*n < 2^31; 1 <= E <= 256;
+ *    E*groups*k < 2^31; 1 <= groups <= 65535.
+ *  - Host threads: calls that use different workspaces (and different saved blobs) may run
+ *    concurrently from different host threads; the library keeps no per-call state outside
+ *    the buffers it is handed.  The exceptions say so in their own comments (ec_route_static's
+ *    shared array, the process-wide ec_profile_* and ec_launch_count).
  */
 #ifndef ECMOE_H_
 #define ECMOE_H_

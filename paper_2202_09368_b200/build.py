@@ -16,7 +16,7 @@ OBJ = os.path.join(HERE, "_build")
 SOURCES = ["api.cu", "routing.cu", "capped.cu", "gemm_simt.cu", "gemm_tc.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-         "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DECMOE_BUILD"]
+         "-Xcompiler", "-fPIC", "-DECMOE_BUILD"]
 
 
 def _newer(src_list, target):

@@ -30,6 +30,7 @@ ec_status check_cfg(const ec_config* c, Dims* D) {
   if (c->n * c->groups >= ((int64_t)1 << 31) || c->E > 256 || c->groups > 65535) return EC_ERR_UNSUPPORTED;
   const size_t eb = esize(c->dtype);
   if ((c->d_model * eb) % 16 || (c->d_ff * eb) % 16) return EC_ERR_UNSUPPORTED;
+  if (c->d_model > (1 << 22) - 64 || c->d_ff > (1 << 22) - 64) return EC_ERR_UNSUPPORTED;   // column tiles of the FMA kernels sit on grid.y
   const int64_t k = ec_capacity(c);
   if (k < 1) return EC_ERR_INVALID_ARG;
   if ((int64_t)c->E * k * c->groups >= ((int64_t)1 << 31)) return EC_ERR_UNSUPPORTED;

@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
   const int b = blockIdx.z;
   const TA* A = (const TA*)g.A + (int64_t)b * g.batch_a;
   const TB* B = (const TB*)g.B + (int64_t)b * g.batch_b;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;     // row tiles on grid.x: M (tokens) is the dimension without a limit
   const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
   float acc[TM][TN];
 #pragma unroll
@@ -106,7 +106,8 @@ static void dispatch_c(const GemmArgs& g, dim3 grid, cudaStream_t st) {
 }
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st) {
-  const dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batches);
+  const dim3 grid((g.M + BM - 1) / BM, (g.N + BN - 1) / BN, g.batches);
+  if (grid.y > 65535u || grid.z > 65535u) return cudaErrorInvalidConfiguration;
   if (g.a_dtype == 0 && g.b_dtype == 0) dispatch_c<float, float>(g, grid, st);
   else if (g.a_dtype == 0) dispatch_c<float, bf16>(g, grid, st);
   else if (g.b_dtype == 0) dispatch_c<bf16, float>(g, grid, st);

@@ -45,6 +45,7 @@
 
 #include <cuda.h>
 #include <cudaTypedefs.h>
+#include <atomic>
 #include <mutex>
 #include <type_traits>
 #include <string.h>
@@ -706,6 +707,8 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
 // tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
 // streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
 int pick_bn(const TcGemmArgs& g, int pairs) {
+  // Eq. 2's softmax runs over all N = E columns of a row inside one tile's epilogue: the tile must hold them all
+  if (g.epi == EPI_SOFTMAX) return g.N > 128 ? 256 : (g.N > 64 ? 128 : 64);
   if (g.M > BM && g.N >= 512 && g.K >= kWideMinK && g.epi == EPI_STORE) {
     // waves of tiles over the CTA pairs, a 512-column tile counted as 1.92 of a 256-column one (its saving in
     // fill less its epilogue in the open): padding of N to 512 and a thinner last wave can cost more than that
@@ -737,14 +740,17 @@ cudaError_t launch_one(const CUtensorMap& ta, const CUtensorMap& tb, const CUten
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    static int max_pairs[64] = {};                   // pairs the device can hold at once, per device
+    // pairs the device can hold at once, per device; host threads may race to fill an entry, with the same value
+    static std::atomic<int> max_pairs[64];
     if (dev >= 0 && dev < 64) {
-      if (max_pairs[dev] == 0) {
+      int mp = max_pairs[dev].load(std::memory_order_relaxed);
+      if (mp == 0) {
         cfg.gridDim = dim3(2 * groups);
         int nc = 0;
-        if (cudaOccupancyMaxActiveClusters(&nc, kern, &cfg) == cudaSuccess && nc > 0) max_pairs[dev] = nc; else max_pairs[dev] = groups;
+        mp = (cudaOccupancyMaxActiveClusters(&nc, kern, &cfg) == cudaSuccess && nc > 0) ? nc : groups;
+        max_pairs[dev].store(mp, std::memory_order_relaxed);
       }
-      if (max_pairs[dev] < groups) groups = max_pairs[dev];
+      if (mp < groups) groups = mp;
     }
   }
   if (p.total_tiles < groups) groups = p.total_tiles;

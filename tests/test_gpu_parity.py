@@ -87,6 +87,29 @@ def test_routing_large_k_and_many_experts(n, E, c):
     check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
 
 
+@pytest.mark.parametrize("n,E,groups", [(128, 256, 1), (64, 256, 2), (100, 200, 1), (128, 136, 1), (512, 256, 1)])
+def test_gate_with_more_experts_than_one_column_tile_and_few_rows(n, E, groups):
+    """E in (128, 256] with at most 128 token rows: the softmax of Eq. 2 still has to see all E logits of a row in one tile."""
+    d = 64
+    li = IN.make_layer_inputs(groups * n, d, 8, E, BF16, seed=7, with_grad=False)
+    cfg = B.make_config(n, d, 8, E, 2.0 * E / 8, BF16, groups=groups)     # k = n / 4 tokens per expert and group
+    r = B.ec_route(cfg, li.X.cuda(), li.Wg.cuda())
+    S = to_np(r.S)
+    assert rel_err(S, O.gate(to_np(li.X), to_np(li.Wg))) <= TOL[BF16]
+    np.testing.assert_allclose(S.sum(axis=1), 1.0, atol=1e-5)
+    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+
+
+def test_read_status_maps_the_status_word():
+    """ec_read_status only reads the first word of the workspace: 0 is EC_OK, 5 a bounded wait that expired, anything
+    else is reported as a CUDA error.  No kernel is involved."""
+    ws = torch.zeros(1024, dtype=torch.int32, device="cuda")
+    for word, want in ((0, B.EC_OK), (5, B.EC_ERR_TIMEOUT), (7, B.EC_ERR_CUDA), (4, B.EC_ERR_CUDA)):
+        ws[0] = word
+        assert B.ec_read_status(ws) == want
+    assert B.lib().ec_read_status(None, None) == B.EC_ERR_INVALID_ARG
+
+
 def test_run_to_run_determinism():
     n, d, dff, E = 1024, 128, 256, 8
     li = IN.make_layer_inputs(n, d, dff, E, BF16, seed=5)

@@ -24,7 +24,10 @@ BF16 = torch.bfloat16
 
 
 @pytest.mark.parametrize("n,E", [(4096, 8), (4096, 32), (4096, 128), (4096, 256), (16384, 32), (16384, 256),
-                                 (65536, 8), (65536, 128)])
+                                 (65536, 8), (65536, 128),
+                                 # the largest groups of the stress grid: k = 65536 .. 2048, sixteen sort tiles and four
+                                 # global bitonic levels at E = 8, eight expert chunks at E = 256
+                                 (262144, 8), (262144, 32), (262144, 128), (262144, 256)])
 def test_routing_only_chain_identity_experts(n, E):
     d, c = 1024, 2.0
     li = IN.make_layer_inputs(n, d, 8, E, BF16, seed=0, with_grad=False)
@@ -46,7 +49,8 @@ def test_routing_only_chain_identity_experts(n, E):
     X_out = B.ec_unshuffle(cfg, X_e, r.G, r.row_ptr, r.slots)
     G = to_np(r.G).reshape(-1)
     ref = np.zeros((n, d))
-    np.add.at(ref, I.reshape(-1), G[:, None] * Xn[I.reshape(-1)])          # fp64 sum over the slots of each token
+    for i in range(E):                                                     # fp64 sum over the slots of each token, Eq. 4;
+        ref[I[i]] += G[i * k:(i + 1) * k, None] * Xn[I[i]]                 # an expert's tokens are distinct
     got = to_np(X_out)
     scale = np.sqrt(np.mean(ref ** 2))
     assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-6 * scale)      # one bf16 rounding
