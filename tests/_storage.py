@@ -19,3 +19,29 @@ def round_bf16(x):
 def bf16_store(name, x):
     """`store=` hook for oracle.forward / oracle.backward: the tensors of BF16_STORED are rounded where they are kept."""
     return round_bf16(x) if name in BF16_STORED else x
+
+
+def half_ulp_bf16(x):
+    """Half the spacing of bfloat16 numbers around x (8 significand bits): the most one rounding can move x."""
+    _, e = np.frexp(np.asarray(x, np.float64))
+    return np.ldexp(1.0, e - 9)
+
+
+class Bf16Recorder:
+    """`store=` hook like bf16_store that also keeps what every rounded tensor was BEFORE it was rounded
+    (per-expert tensors in call order), so a test can tell apart the two things bf16 storage does to an output:
+    the error its operands carried in (pre - reference) and its own final rounding (at most half_ulp_bf16(pre))."""
+
+    def __init__(self):
+        self.pre = {}
+
+    def __call__(self, name, x):
+        if name not in BF16_STORED:
+            return x
+        self.pre.setdefault(name, []).append(np.array(x, np.float64))
+        return round_bf16(x)
+
+    def before(self, name, like):
+        """The unrounded version of tensor `name`, shaped like `like` (the stack over experts where it is per expert)."""
+        got = self.pre[name]
+        return got[0] if len(got) == 1 and got[0].shape == like.shape else np.stack(got)
