@@ -111,16 +111,38 @@ def workload_desc(name, groups=1, cap_b=0, cap_iters=100):
             f"{how}")
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches
-# of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_cfg4e4.md: 625.2 MB at 4 experts of
-# the 8B/64E shape.  Operands, outputs and weights all grow with the number of experts, so a launch at E experts
-# moves E/4 times as much.  None for shapes that were not captured.
-GEMM_TRAFFIC_PER_EXPERT = {"cfg4": 625.2e6 / 4, "cfg4e4": 625.2e6 / 4}
+GEMM_PROFILE = os.path.join(ROOT, "profiles", "gemm_tc_kernel_cfg4e4.md")
+GEMM_SOURCE = os.path.join(ROOT, "paper_2202_09368_b200", "csrc", "gemm_tc.cu")
+
+
+def source_digest(path=GEMM_SOURCE):
+    import hashlib
+    with open(path, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
 
 
 def gemm_traffic(workload, E):
-    per = GEMM_TRAFFIC_PER_EXPERT.get(workload)
-    return None if per is None else per * E
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per expert-GEMM launch, mean over the six launches of
+    a step, read from the ncu summary under profiles/ (a capture of four experts of the 8B/64E shape: operands,
+    outputs and weights all grow with the number of experts, so a launch at E experts moves E/4 times as much).
+    None for shapes that were not captured, and None when the kernel source is no longer the one that was captured
+    (the summary records a digest of it)."""
+    if workload not in ("cfg4", "cfg4e4") or not os.path.exists(GEMM_PROFILE):
+        return None
+    rd = wr = None
+    digest = None
+    for line in open(GEMM_PROFILE):
+        cells = [c.strip() for c in line.split("|")]
+        if len(cells) > 3 and cells[1] == "dram__bytes_read.sum":
+            rd = [float(c) for c in cells[3:] if c]
+        if len(cells) > 3 and cells[1] == "dram__bytes_write.sum":
+            wr = [float(c) for c in cells[3:] if c]
+        if line.startswith("kernel source digest:"):
+            digest = line.split(":", 1)[1].strip().strip("`")
+    if not rd or not wr or len(rd) != len(wr) or digest != source_digest():
+        return None
+    per_launch_e4 = sum(a + b for a, b in zip(rd, wr)) / len(rd) * 1e6          # the table is in Mbyte
+    return per_launch_e4 * E / 4
 
 
 def layer_flops(n, d, dff, E, c):
@@ -158,23 +180,33 @@ def time_oracle_sample(n, d, dff, E, c, seed=0, budget_s=12.0, groups=1):
     r = O.route(X, Wg, c, groups=groups)
     t_route = time.perf_counter() - t0
     t_sum, experts = 0.0, 0
+    k = r["I"].shape[1]
+    X_out, dX = np.zeros((n, d)), np.zeros((n, d))
+    dG = np.zeros((E, k))
     while experts < E and (experts == 0 or t_route + t_sum < budget_s):
         i = experts
         W1_i, W2_i = weights(IN.TID_W1, i, d), weights(IN.TID_W2, i, dff)      # generation is not timed
         t0 = time.perf_counter()
-        I_i, G_i = r["I"][i], r["G"][i]
-        X_in = X[I_i]
+        I_i, G_i = r["I"][i:i + 1], r["G"][i:i + 1]
+        X_in = X[I_i[0]]
         Z, H, X_e = O.expert_ffn(X_in, W1_i, W2_i)
-        dX_e = G_i[:, None] * dY[I_i]
-        dG = np.einsum("jd,jd->j", dY[I_i], X_e)
-        O.expert_ffn_backward(dX_e, X_in, Z, H, W1_i, W2_i)
+        X_out += O.combine(X_e[None], G_i, I_i, n)                             # Eq. 4, this expert's share
+        dX_e = G_i[0][:, None] * dY[I_i[0]]
+        dG[i] = np.einsum("jd,jd->j", dY[I_i[0]], X_e)
+        _, _, dX_in, _, _ = O.expert_ffn_backward(dX_e, X_in, Z, H, W1_i, W2_i)
+        O.add_slot_rows(dX, I_i, dX_in[None])
         t_sum += time.perf_counter() - t0
         experts += 1
+    t0 = time.perf_counter()                                                   # the gate's backward, in full
+    _, dL = O.softmax_backward(r["S"], r["I"], dG)
+    dWg = X.T @ dL
+    dX += dL @ Wg.T
+    t_gate = time.perf_counter() - t0
     t_exp = t_sum / experts
-    total = t_route + E * t_exp
+    total = t_route + E * t_exp + t_gate
     what = (f"oracle (numpy fp64) on n={n} d={d} d'={dff} E={E} c={c}: routing in full ({t_route:.2f} s) + "
-            f"{experts} of {E} experts forward+backward ({t_exp:.2f} s each), expert part extrapolated x{E}; "
-            f"combine and gate backward not included")
+            f"{experts} of {E} experts forward+backward with their share of the combine ({t_exp:.2f} s each), expert part "
+            f"extrapolated x{E}; gate backward in full ({t_gate:.2f} s)")
     return n / total, threads, what
 
 
@@ -183,13 +215,16 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    # every step is a bounded sample of the workload (seconds of CPU work); at most two are run however many were asked for
+    ran = max(1, min(args.steps, 2))
     vals = []
-    for _ in range(max(1, min(args.steps, 2))):          # bounded: each step is seconds of CPU work
+    for _ in range(ran):
         v, threads, what = time_oracle_sample(n, d, dff, E, c, groups=args.groups)
         vals.append(v)
     v = sum(vals) / len(vals)
     out = {"impl": "reference", "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": v, "unit": "tokens/s",
-           "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * n / v,
+           "n_gpus": args.gpus, "steps": ran, "steps_requested": args.steps, "warmup": 0, "ms_per_step": 1e3 * n / v,
+           "ms_per_step_is": "extrapolated: the time of one whole step at the sampled rate, not the time the sample took",
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
            "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters)},
            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
@@ -262,19 +297,28 @@ def run_gpu(args):
             step()
         eager_step, step = step, graph.replay
         step(); torch.cuda.synchronize()
-    # ---- timed region: K steps, device timed, max over ranks
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    l0 = B.ec_launch_count()
-    with ClockSampler(local) as clocks:
-        ev0.record()
-        for _ in range(args.steps):
-            step()
-        ev1.record()
+    # ---- timed region: K steps, device timed, max over ranks; repeated R times in this run so that the line can say
+    # how much one region differs from the next on this machine (the SM clock under the power cap moves by several
+    # percent).  `value` is the median region; the clock sampled during each region is reported beside its time.
+    repeats = max(1, args.repeats)
+    region_ms, region_mhz, launches, all_rows = [], [], 0, []
+    for rep in range(repeats):
         barrier()
-    launches = B.ec_launch_count() - l0
-    ms_total = aggregate_max(ev0.elapsed_time(ev1), dev)
-    ms_step = ms_total / args.steps
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = B.ec_launch_count()
+        with ClockSampler(local) as clocks:
+            ev0.record()
+            for _ in range(args.steps):
+                step()
+            ev1.record()
+            barrier()
+        launches = B.ec_launch_count() - l0
+        region_ms.append(aggregate_max(ev0.elapsed_time(ev1), dev) / args.steps)
+        region_mhz.append(clocks.summary()["sm_mhz"])
+        all_rows += clocks.rows
+    clocks.rows = all_rows                                         # the summary on the line covers every region
+    order = sorted(range(repeats), key=lambda i: region_ms[i])
+    ms_step = region_ms[order[repeats // 2]]
     assert B.ec_read_status(ws) == B.EC_OK
 
     # ---- per-stage times (CUDA events recorded by the library on the launching stream).  Steps are
@@ -348,6 +392,9 @@ def run_gpu(args):
         out = {
             "metric": "ec_moe_layer_tokens_per_s_fwd_bwd", "value": world * n / (ms_step * 1e-3), "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
+            "regions": {"count": repeats, "steps_each": args.steps, "ms_per_step": [round(v, 4) for v in region_ms],
+                        "sm_mhz": region_mhz, "median_ms": round(ms_step, 4), "best_ms": round(min(region_ms), 4),
+                        "ms_x_mhz": [round(a * b, 1) if b else None for a, b in zip(region_ms, region_mhz)]},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
@@ -521,7 +568,8 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=40, help="steps per timed region")
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions per run; the line reports the median one")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(WORKLOADS))

@@ -137,6 +137,38 @@ def expert_ffn_backward(dX_e_i, X_in_i, Z_i, H_i, W1_i, W2_i, gelu_variant: str 
     return dW1, dW2, dX_in, store("dH", dH), dZ
 
 
+def combine(X_e, G, I, n: int):
+    """Eq. 4: X_out[t, :] = sum over the slots (i, j) with I[i, j] = t of G[i, j] * X_e[i, j, :], experts in
+    ascending order; rows of tokens that no expert chose stay zero."""
+    e, k = I.shape
+    X_out = np.zeros((n, X_e.shape[2]), F64)
+    for i in range(e):
+        for j in range(k):
+            X_out[I[i, j]] += G[i, j] * X_e[i, j]
+    return X_out
+
+
+def softmax_backward(S, I, dG, store=_keep):
+    """Chain rule through Eq. 2 with I held constant: dS[t, i] = dG[i, j] where I[i, j] = t (else 0), and the
+    softmax Jacobian per token row, dL = S * (dS - <dS, S>)."""
+    n, e = S.shape
+    dS = np.zeros((n, e), F64)
+    for i in range(e):
+        dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
+    dS = store("dS", dS)
+    dL = store("dL", S * (dS - (dS * S).sum(axis=1, keepdims=True)))
+    return dS, dL
+
+
+def add_slot_rows(dX, I, dX_in):
+    """Chain rule through Eq. 3's X_in = P . X: every slot's gradient row goes back to its token (in place)."""
+    e, k = I.shape
+    for i in range(e):
+        for j in range(k):
+            dX[I[i, j]] += dX_in[i, j]
+    return dX
+
+
 def capped_assignment(S, k: int, b: int, lam: float = 1e-3, iters: int = 100):
     """Section 3.3 (expert choice with at most b experts per token): the matrix A [e, n] of
 
@@ -236,11 +268,7 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
     Z = np.stack([p[0] for p in per_expert])               # [e, k, d']
     H = np.stack([p[1] for p in per_expert])               # [e, k, d']
     X_e = np.stack([p[2] for p in per_expert])             # [e, k, d]
-    X_out = np.zeros((n, d), F64)                          # Eq. 4, experts in ascending order
-    for i in range(e):
-        for j in range(k):
-            X_out[I[i, j]] += G[i, j] * X_e[i, j]
-    X_out = store("X_out", X_out)
+    X_out = store("X_out", combine(X_e, G, I, n))          # Eq. 4
     r.update(X_in=X_in, Z=Z, H=H, X_e=X_e, X_out=X_out)
     return r
 
@@ -266,17 +294,9 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     dX_in = np.stack([p[2] for p in per_expert])           # [e, k, d]
     dH = np.stack([p[3] for p in per_expert])
     dZ = np.stack([p[4] for p in per_expert])
-    dS = np.zeros((n, e), F64)
-    for i in range(e):
-        dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
-    dS = store("dS", dS)
-    dL = store("dL", S * (dS - (dS * S).sum(axis=1, keepdims=True)))   # softmax Jacobian, per token row
+    dS, dL = softmax_backward(S, I, dG, store)
     dWg = store("dWg", X.T @ dL)
-    dX = dL @ Wg.T
-    for i in range(e):
-        for j in range(k):
-            dX[I[i, j]] += dX_in[i, j]
-    dX = store("dX", dX)
+    dX = store("dX", add_slot_rows(dL @ Wg.T, I, dX_in))
     return dict(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2, dX_e=dX_e, dG=dG, dH=dH, dZ=dZ,
                 dX_in=dX_in, dS=dS, dL=dL)
 
