@@ -79,12 +79,13 @@ def topk(S, k: int):
 def inverse_index(I, n: int):
     """Index form of P = Onehot(I) (Eq. 2) read by token: for token t, the flat
     slot ids i*k+j with I[i, j] = t, in ascending order (hence ascending expert).
-    Returns row_ptr [n+1] and slots [e*k]."""
+    Returns row_ptr [n+1] and slots [number of filled slots] (e*k with expert choice)."""
     I = np.asarray(I)
     e, k = I.shape
     flat = I.reshape(-1)
-    order = np.argsort(flat, kind="stable")          # ascending token, then ascending slot id
-    counts = np.bincount(flat, minlength=n)
+    filled = np.flatnonzero(flat >= 0)               # every slot with expert choice; token choice may leave slots empty (-1)
+    order = filled[np.argsort(flat[filled], kind="stable")]      # ascending token, then ascending slot id
+    counts = np.bincount(flat[filled], minlength=n)
     row_ptr = np.zeros(n + 1, np.int64)
     row_ptr[1:] = np.cumsum(counts)
     return row_ptr, order.astype(np.int64)
@@ -144,7 +145,8 @@ def combine(X_e, G, I, n: int):
     X_out = np.zeros((n, X_e.shape[2]), F64)
     for i in range(e):
         for j in range(k):
-            X_out[I[i, j]] += G[i, j] * X_e[i, j]
+            if I[i, j] >= 0:                               # empty slots (token choice only) hold no token
+                X_out[I[i, j]] += G[i, j] * X_e[i, j]
     return X_out
 
 
@@ -154,7 +156,8 @@ def softmax_backward(S, I, dG, store=_keep):
     n, e = S.shape
     dS = np.zeros((n, e), F64)
     for i in range(e):
-        dS[I[i], i] = dG[i]                                # tokens of one expert are distinct
+        f = I[i] >= 0
+        dS[I[i][f], i] = dG[i][f]                          # tokens of one expert are distinct
     dS = store("dS", dS)
     dL = store("dL", S * (dS - (dS * S).sum(axis=1, keepdims=True)))
     return dS, dL
@@ -165,7 +168,8 @@ def add_slot_rows(dX, I, dX_in):
     e, k = I.shape
     for i in range(e):
         for j in range(k):
-            dX[I[i, j]] += dX_in[i, j]
+            if I[i, j] >= 0:
+                dX[I[i, j]] += dX_in[i, j]
     return dX
 
 
@@ -201,12 +205,38 @@ def capped_assignment(S, k: int, b: int, lam: float = 1e-3, iters: int = 100):
     return np.exp(L)
 
 
+def token_choice(S, capacity: int, top: int = 2):
+    """The conventional routing Section 3.1 contrasts expert choice with, on the same scores: every token
+    independently picks its `top` highest-scoring experts (equal scores: the lower expert index), and an expert,
+    whose buffer holds `capacity` tokens, takes the requests in token order and drops what no longer fits.
+    Returns I [e, capacity] (token per slot in order of arrival, -1 = empty slot), G [e, capacity] (S at the
+    filled slots, 0 at the empty ones), load [e] (slots filled) and requested [e] (requests before dropping)."""
+    S = np.asarray(S)
+    n, e = S.shape
+    I = np.full((e, capacity), -1, np.int64)
+    G = np.zeros((e, capacity), S.dtype)
+    load = np.zeros(e, np.int64)
+    requested = np.zeros(e, np.int64)
+    for t in range(n):
+        order = np.argsort(-S[t], kind="stable")           # descending score, equal scores by ascending expert
+        for i in order[:top]:
+            requested[i] += 1
+            if load[i] < capacity:
+                I[i, load[i]] = t
+                G[i, load[i]] = S[t, i]
+                load[i] += 1
+    return G, I, load, requested
+
+
 def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3,
-          cap_iters: int = 100):
+          cap_iters: int = 100, router: str = "expert"):
     """Eq. 1-2: S, G, I and the token->slot inverse index.
 
     cap_b > 0 (Section 3.3): the indices are TopK(A, k) of the capped assignment A instead of TopK(S^T, k);
     the gate weights stay G[i, j] = S[I[i, j], i].  The result then also holds A as [n, e].
+
+    router = "token": the token-choice contrast of token_choice() with two experts per token and buffers of
+    k = n*c/e slots; I then holds -1 in empty slots, and the result also has load and requested, [groups, e].
 
     groups > 1 (the paper's Limitations section: route several groups of tokens independently):
     X holds `groups` blocks of n rows; Eq. 1-2 are applied to each block on its own with k = n*c/e,
@@ -219,6 +249,15 @@ def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap
     n = N // groups
     k = capacity(n, c, e)
     S = gate(X, Wg) if S_override is None else np.asarray(S_override, F64)
+    if router == "token":
+        parts = [token_choice(S[g * n:(g + 1) * n], k) for g in range(groups)]
+        G = np.concatenate([p[0] for p in parts], axis=1)
+        I = np.concatenate([np.where(p[1] >= 0, p[1] + g * n, -1) for g, p in enumerate(parts)], axis=1)
+        row_ptr, slots = inverse_index(I, N)
+        return dict(k=k * groups, S=S, G=G, I=I, row_ptr=row_ptr, slots=slots,
+                    load=np.stack([p[2] for p in parts]), requested=np.stack([p[3] for p in parts]))
+    if router != "expert":
+        raise ValueError(router)
     if cap_b:
         A = np.concatenate([capped_assignment(S[g * n:(g + 1) * n], k, cap_b, cap_lambda, cap_iters).T
                             for g in range(groups)])
@@ -234,14 +273,16 @@ def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap
 
 
 def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
-            store=_keep, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3, cap_iters: int = 100):
+            store=_keep, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3, cap_iters: int = 100,
+            router: str = "expert"):
     """Eq. 1-4.  Returns every intermediate.
 
     S_override replaces the gate output (the routing is then taken from it);
     I_override additionally fixes the index matrix (G is read from S at I).
     Both exist so that later stages can be compared on identical routing.
 
-    cap_b > 0 routes with the capped assignment of Section 3.3 (see route()).
+    cap_b > 0 routes with the capped assignment of Section 3.3, router = "token" with the token-choice
+    contrast of Section 3.1 (see route()); empty slots then hold zero rows throughout.
 
     `store(name, array)` is handed EVERY named tensor the layer produces after the routing
     (X_in, Z, H, X_e, X_out here; dX_e, dG, dH, dZ, dW1, dW2, dX_in, dS, dL, dWg, dX in backward()),
@@ -255,15 +296,18 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
     W1 = np.asarray(W1, F64); W2 = np.asarray(W2, F64)
     n, d = X.shape
     e = Wg.shape[1]
-    r = route(X, Wg, c, S_override, groups, cap_b, cap_lambda, cap_iters)
+    r = route(X, Wg, c, S_override, groups, cap_b, cap_lambda, cap_iters, router)
     k, S = r["k"], r["S"]
     if I_override is not None:
         I = np.asarray(I_override, np.int64)
-        G = np.stack([S[I[i], i] for i in range(e)])
+        G = np.stack([np.where(I[i] >= 0, S[I[i], i], 0.0) for i in range(e)])
         row_ptr, slots = inverse_index(I, n)
         r.update(I=I, G=G, row_ptr=row_ptr, slots=slots)
     I, G = r["I"], r["G"]
-    X_in = store("X_in", X[I])                             # Eq. 3: X_in = P . X,  [e, k, d]
+    X_in = X[I]                                            # Eq. 3: X_in = P . X,  [e, k, d]
+    if (I < 0).any():
+        X_in[I < 0] = 0.0                                  # an empty slot (token choice only) holds a zero row
+    X_in = store("X_in", X_in)
     per_expert = [expert_ffn(X_in[i], W1[i], W2[i], gelu_variant, store) for i in range(e)]
     Z = np.stack([p[0] for p in per_expert])               # [e, k, d']
     H = np.stack([p[1] for p in per_expert])               # [e, k, d']
@@ -285,6 +329,8 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     X_in, Z, H, X_e = fwd["X_in"], fwd["Z"], fwd["H"], fwd["X_e"]
     k = I.shape[1]
     dY = dX_out[I]                                         # [e, k, d] rows of dX_out seen by each slot
+    if (I < 0).any():
+        dY[I < 0] = 0.0                                    # empty slots see no token
     dX_e = store("dX_e", G[:, :, None] * dY)               # Eq. 4 w.r.t. X_e
     dG = store("dG", np.einsum("ijd,ijd->ij", dY, X_e))    # Eq. 4 w.r.t. G
     per_expert = [expert_ffn_backward(dX_e[i], X_in[i], Z[i], H[i], W1[i], W2[i], gelu_variant, store)
