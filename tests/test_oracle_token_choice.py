@@ -112,7 +112,7 @@ def test_dropped_tokens_get_what_their_surviving_experts_give_them():
 
 @pytest.mark.parametrize("variant", ["erf", "tanh"])
 def test_backward_matches_finite_differences_with_token_choice(variant):
-    n, d, dff, E, c = 40, 6, 10, 4, 1.5
+    n, d, dff, E, c = 40, 6, 10, 4, 1.9      # buffers of 19 slots for 17 to 25 requests: drops and empty slots
     X, Wg, W1, W2, dY = mk(n, d, dff, E, seed=11)
     f = O.forward(X, Wg, W1, W2, c, variant, router="token")
     b = O.backward(X, Wg, W1, W2, dY, f, variant)
