@@ -565,6 +565,80 @@ def run_sweep(args):
                       "cases": cases}))
 
 
+# ----------------------------------------------------------------------------------- token-choice contrast
+def run_contrast(args):
+    """Expert choice next to the token-choice top-2 routing it is contrasted with (Section 3.1, Section 4.2), on
+    identical synthetic inputs: step time (forward + backward, median of the timed regions), expert loads, dropped
+    requests.  Four runs of the same layer:
+      expert_choice          the paper's method, k = n*c/e slots per expert, all filled;
+      token_top2             two experts per token, buffers of the same k slots, requests beyond them dropped;
+      token_top2_no_drop     buffers enlarged to what the fullest expert asks for, nothing dropped; the GEMMs skip empty slots;
+      fixed_shape_no_drop    what an implementation with fixed buffer shapes pays for those enlarged buffers: every
+                             slot of every buffer is computed (timed as expert choice at that buffer size).
+    `--expert-skew` gives some experts a popularity offset, standing in for the imbalance of a trained gate."""
+    import torch
+    from paper_2202_09368_b200 import binding as B
+    from paper_2202_09368_b200 import inputs as IN
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dev = torch.device("cuda")
+    n, d, dff, E, c = WORKLOADS[args.workload]
+    bf, chunk = torch.bfloat16, 1 << 26
+    li = IN.make_layer_inputs(n, d, 8, E, bf, 0, device=dev, with_grad=False, expert_skew=args.expert_skew)
+    X, Wg = li.X, li.Wg
+    W1 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(d), 0, IN.TID_W1, bf, dev, chunk)
+    W2 = IN.normal_tensor((E, d, dff), 1.0 / math.sqrt(dff), 0, IN.TID_W2, bf, dev, chunk)
+    dY = IN.normal_tensor((n, d), 1.0, 0, IN.TID_DXOUT, bf, dev, chunk)
+    X_out = torch.empty_like(X)
+    grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
+
+    def timed(cfg):
+        ws, saved = B.alloc_workspace(cfg, dev), B.alloc_saved(cfg, dev)
+
+        def step():
+            B.ec_moe_forward(cfg, X, Wg, W1, W2, X_out, saved, ws)
+            B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, grads, ws)
+        for _ in range(max(3, args.warmup)):
+            step()
+        assert B.ec_read_status(ws) == B.EC_OK
+        ms = []
+        for _ in range(max(1, args.repeats)):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(args.steps):
+                step()
+            b_.record()
+            torch.cuda.synchronize()
+            ms.append(a.elapsed_time(b_) / args.steps)
+        assert B.ec_read_status(ws) == B.EC_OK
+        v = B.saved_view(cfg, saved)
+        per_token = torch.bincount((v["row_ptr"][1:] - v["row_ptr"][:-1]).long()).tolist()
+        out = {"ms_per_step": round(sorted(ms)[len(ms) // 2], 4), "best_ms": round(min(ms), 4), "slots_per_expert": B.ec_capacity(cfg),
+               "tokens_by_number_of_experts": per_token}
+        if cfg.router:
+            load, req = v["load"].view(-1).tolist(), v["requested"].view(-1).tolist()
+            k = B.ec_capacity(cfg)
+            out.update({"requested_min_median_max": [min(req), sorted(req)[len(req) // 2], max(req)],
+                        "fullest_expert_over_buffer": round(max(req) / k, 3), "experts_over_their_buffer": sum(r > k for r in req),
+                        "requests_dropped": round(1.0 - sum(load) / sum(req), 4), "filled_slots": sum(load)})
+        del ws, saved
+        return out, (v["requested"].max().item() if cfg.router else None)
+
+    res = {}
+    res["expert_choice"], _ = timed(B.make_config(n, d, dff, E, c, bf))
+    res["token_top2"], fullest = timed(B.make_config(n, d, dff, E, c, bf, router="token"))
+    c_big = (fullest + 0.5) * E / n                                # buffers of exactly what the fullest expert asked for
+    res["token_top2_no_drop"], _ = timed(B.make_config(n, d, dff, E, c_big, bf, router="token"))
+    res["fixed_shape_no_drop"], _ = timed(B.make_config(n, d, dff, E, c_big, bf))
+    ec = res["expert_choice"]["ms_per_step"]
+    print(json.dumps({"metric": "ec_vs_token_choice_step_time", "unit": "ms per forward+backward step (median region)",
+                      "config": {"workload": workload_desc(args.workload), "expert_skew": args.expert_skew,
+                                 "data": "synthetic; a popularity offset per expert stands in for a trained gate's imbalance",
+                                 "regions": args.repeats, "steps_each": args.steps},
+                      "runs": res,
+                      "step_time_over_expert_choice": {k_: round(v_["ms_per_step"] / ec, 3) for k_, v_ in res.items()}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -581,8 +655,12 @@ def main():
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")
+    ap.add_argument("--contrast", action="store_true", help="expert choice beside token-choice top-2 routing on identical inputs")
+    ap.add_argument("--expert-skew", type=float, default=0.05, help="with --contrast: popularity offset of the experts' gate logits")
     args = ap.parse_args()
-    if args.sweep:
+    if args.contrast:
+        run_contrast(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.routing:
         run_routing(args)

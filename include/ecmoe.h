@@ -60,6 +60,14 @@ typedef enum {
 
 typedef enum { EC_F32 = 0, EC_BF16 = 1 } ec_dtype;
 typedef enum { EC_GELU_ERF = 0, EC_GELU_TANH = 1 } ec_gelu;
+/* Who chooses: EC_ROUTER_EXPERT_CHOICE is the paper's method (Section 3.2).  EC_ROUTER_TOKEN_TOP2 is the conventional
+ * routing Section 3.1 contrasts it with, provided as a synthetic contrast workload on the same layer: every token picks
+ * its two highest-scoring experts (equal scores: the lower expert), an expert's buffer holds k = n*c/e tokens (Eq. 1's
+ * formula read as the buffer size), takes requests in token order and drops what does not fit.  Slots are then filled
+ * in order of arrival, I holds -1 and G holds 0 in empty slots, tokens have 0, 1 or 2 experts, and everything after
+ * the routing (Eq. 3-4, the backward pass with the choices held constant) is the same code on those slots; the
+ * tensor-core GEMMs skip the tiles and k-blocks that hold only empty slots (with groups = 1). */
+typedef enum { EC_ROUTER_EXPERT_CHOICE = 0, EC_ROUTER_TOKEN_TOP2 = 1 } ec_router;
 
 /* One layer call.  Plain data, passed by pointer, never retained. */
 typedef struct {
@@ -75,6 +83,8 @@ typedef struct {
   int32_t cap_b;     /* b: bound on the column sums of A; needs E*k <= n*b                      */
   int32_t cap_iters; /* rounds of Dykstra's algorithm (the paper: at most 100), >= 1            */
   double cap_lambda; /* weight of the entropy term (the paper: 0.001), > 0                      */
+  int32_t router;    /* ec_router; the token-choice contrast needs cap_b = 0 and E >= 2         */
+  int32_t reserved;  /* 0                                                                       */
 } ec_config;
 
 /* Views into the forward->backward blob (device pointers), for inspection and tests. */
@@ -88,6 +98,8 @@ typedef struct {
   void* Z;          /* [E, k, d'] X_in[i] . W1[i]                                      */
   void* H;          /* [E, k, d'] GeLU(Z)                                              */
   float* X_e;       /* [E, k, d]  expert outputs H[i] . W2[i]^T, fp32 on both paths    */
+  int32_t* load;      /* [groups, E] slots filled per expert (EC_ROUTER_TOKEN_TOP2 only, else NULL)   */
+  int32_t* requested; /* [groups, E] tokens that asked for the expert, before dropping (same)         */
 } ec_saved_ptrs;
 
 /* Eq. 1: k = floor(n*c/E), per routing group.  Returns -1 when cfg is NULL or k falls outside [1, n]. */
@@ -120,6 +132,17 @@ ec_status ec_saved_view(const ec_config* cfg, void* saved, ec_saved_ptrs* out);
 ec_status ec_route(const ec_config* cfg, const void* X, const void* Wg, float* S, int32_t* I,
                    float* G, int32_t* row_ptr, int32_t* slots, void* ws, size_t ws_bytes,
                    void* cuda_stream);
+
+/*
+ * The token-choice contrast routing (see ec_router) on its own; cfg->router must be EC_ROUTER_TOKEN_TOP2 (ec_route and
+ * ec_route_static refuse such a cfg with EC_ERR_INVALID_ARG: they have nowhere to put the loads).  Outputs as for
+ * ec_route, with -1 / 0 in the empty slots of I / G and only the first row_ptr[n] entries of `slots` written, plus
+ * load and requested, [groups, E] int32 each: slots filled per expert and tokens that asked for it.  max(requested) / k
+ * is how far the fullest expert is over its buffer (Section 3.1's over-capacity ratio, plus one).
+ */
+ec_status ec_route_token_choice(const ec_config* cfg, const void* X, const void* Wg, float* S, int32_t* I,
+                                float* G, int32_t* row_ptr, int32_t* slots, int32_t* load,
+                                int32_t* requested, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * Section 3.3 on its own: the assignment A of

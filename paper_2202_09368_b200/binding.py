@@ -18,24 +18,26 @@ _lib = None
 EC_OK, EC_ERR_INVALID_ARG, EC_ERR_UNSUPPORTED, EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT = range(6)
 EC_F32, EC_BF16 = 0, 1
 EC_GELU_ERF, EC_GELU_TANH = 0, 1
+EC_ROUTER_EXPERT_CHOICE, EC_ROUTER_TOKEN_TOP2 = 0, 1
 
 EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view", "ec_route",
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
            "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
-           "ec_forward_only_workspace_bytes", "ec_capped_assignment"]
+           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice"]
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class ec_config(C.Structure):
     _fields_ = [("n", C.c_int64), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32),
                 ("groups", C.c_int32), ("c", C.c_double), ("dtype", C.c_int32), ("gelu", C.c_int32),
-                ("cap_b", C.c_int32), ("cap_iters", C.c_int32), ("cap_lambda", C.c_double)]
+                ("cap_b", C.c_int32), ("cap_iters", C.c_int32), ("cap_lambda", C.c_double),
+                ("router", C.c_int32), ("reserved", C.c_int32)]
 
 
 class ec_saved_ptrs(C.Structure):
     _fields_ = [(name, C.c_void_p) for name in
-                ("S", "I", "G", "row_ptr", "slots", "X_in", "Z", "H", "X_e")]
+                ("S", "I", "G", "row_ptr", "slots", "X_in", "Z", "H", "X_e", "load", "requested")]
 
 
 class EcError(RuntimeError):
@@ -60,6 +62,8 @@ def lib():
         L.ec_saved_view.restype = C.c_int; L.ec_saved_view.argtypes = [P, V, C.POINTER(ec_saved_ptrs)]
         L.ec_route.restype = C.c_int
         L.ec_route.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V]
+        L.ec_route_token_choice.restype = C.c_int
+        L.ec_route_token_choice.argtypes = [P, V, V, V, V, V, V, V, V, V, V, C.c_size_t, V]
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
@@ -86,11 +90,13 @@ def status_string(code: int) -> str:
 
 
 def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=1, cap_b=0, cap_iters=100,
-                cap_lambda=1e-3) -> ec_config:
-    """cap_b > 0: at most cap_b experts per token (Section 3.3) with the paper's solver settings as defaults."""
+                cap_lambda=1e-3, router="expert") -> ec_config:
+    """cap_b > 0: at most cap_b experts per token (Section 3.3) with the paper's solver settings as defaults.
+    router = "token": the token-choice top-2 contrast of Section 3.1 with expert buffers of n*c/E slots."""
     dt = {torch.float32: EC_F32, torch.bfloat16: EC_BF16}[dtype]
     return ec_config(int(n), int(d_model), int(d_ff), int(E), int(groups), float(c), dt,
-                     {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu], int(cap_b), int(cap_iters), float(cap_lambda))
+                     {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu], int(cap_b), int(cap_iters), float(cap_lambda),
+                     {"expert": EC_ROUTER_EXPERT_CHOICE, "token": EC_ROUTER_TOKEN_TOP2}[router], 0)
 
 
 def ec_capacity(cfg: ec_config) -> int:
@@ -156,6 +162,8 @@ class Routing:
     G: torch.Tensor
     row_ptr: torch.Tensor
     slots: torch.Tensor
+    load: torch.Tensor | None = None          # token-choice contrast only: slots filled per expert, [groups, E]
+    requested: torch.Tensor | None = None     # and tokens that asked for each expert
 
 
 def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
@@ -173,6 +181,24 @@ def ec_route(cfg, X, Wg, ws=None, out: Routing | None = None) -> Routing:
     ws = alloc_workspace(cfg, dev) if ws is None else ws
     _check(lib().ec_route(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
                           _ptr(out.row_ptr), _ptr(out.slots), _ptr(ws), ws.numel(), _stream()), "ec_route")
+    return out
+
+
+def ec_route_token_choice(cfg, X, Wg, ws=None) -> Routing:
+    """The token-choice contrast routing (cfg.router = token): I holds -1 and G holds 0 in empty slots; only the
+    first row_ptr[-1] entries of `slots` are meaningful."""
+    n, k, dev = total_tokens(cfg), slots_per_expert(cfg), X.device
+    out = Routing(torch.empty(n, cfg.E, dtype=torch.float32, device=dev),
+                  torch.empty(cfg.E, k, dtype=torch.int32, device=dev),
+                  torch.empty(cfg.E, k, dtype=torch.float32, device=dev),
+                  torch.empty(n + 1, dtype=torch.int32, device=dev),
+                  torch.empty(cfg.E * k, dtype=torch.int32, device=dev),
+                  torch.empty(cfg.groups, cfg.E, dtype=torch.int32, device=dev),
+                  torch.empty(cfg.groups, cfg.E, dtype=torch.int32, device=dev))
+    ws = alloc_workspace(cfg, dev) if ws is None else ws
+    _check(lib().ec_route_token_choice(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(out.S), _ptr(out.I), _ptr(out.G),
+                                       _ptr(out.row_ptr), _ptr(out.slots), _ptr(out.load), _ptr(out.requested),
+                                       _ptr(ws), ws.numel(), _stream()), "ec_route_token_choice")
     return out
 
 
@@ -288,7 +314,11 @@ def saved_view(cfg, saved) -> dict:
         return saved[off:off + cnt * esz].view(dtype).view(*shape)
 
     n, E, d, f = total_tokens(cfg), cfg.E, cfg.d_model, cfg.d_ff
-    return dict(S=view(v.S, (n, E), torch.float32, 4), I=view(v.I, (E, k), torch.int32, 4),
+    extra = {}
+    if cfg.router == EC_ROUTER_TOKEN_TOP2:
+        extra = dict(load=view(v.load, (cfg.groups, E), torch.int32, 4),
+                     requested=view(v.requested, (cfg.groups, E), torch.int32, 4))
+    return dict(**extra, S=view(v.S, (n, E), torch.float32, 4), I=view(v.I, (E, k), torch.int32, 4),
                 G=view(v.G, (E, k), torch.float32, 4), row_ptr=view(v.row_ptr, (n + 1,), torch.int32, 4),
                 slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es),
                 Z=view(v.Z, (E, k, f), dt, es), H=view(v.H, (E, k, f), dt, es),

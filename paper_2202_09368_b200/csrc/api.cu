@@ -19,7 +19,7 @@ inline size_t esize(int dtype) { return dtype == EC_F32 ? 4 : 2; }
 // n: all tokens of the call (groups * tokens per group), k: slots per expert (groups * k per group),
 // slots = E * k; ng, kg: the per-group values Eq. 1 is about.
 struct Dims { int64_t n, k, slots, ng, kg; int d, dff, E, groups; int dtype, gelu; size_t eb;
-              int cap_b, cap_iters; double cap_lambda; };
+              int cap_b, cap_iters; double cap_lambda; int router; };
 
 ec_status check_cfg(const ec_config* c, Dims* D) {
   if (!c) return EC_ERR_INVALID_ARG;
@@ -39,14 +39,16 @@ ec_status check_cfg(const ec_config* c, Dims* D) {
     if (c->cap_iters < 1 || !(c->cap_lambda > 0.0)) return EC_ERR_INVALID_ARG;
     if ((int64_t)c->E * k > c->n * (int64_t)c->cap_b) return EC_ERR_INVALID_ARG;     // E*k slots cannot fit under the cap
   }
-  if (D) { D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
+  if (c->router != EC_ROUTER_EXPERT_CHOICE && c->router != EC_ROUTER_TOKEN_TOP2) return EC_ERR_INVALID_ARG;
+  if (c->router == EC_ROUTER_TOKEN_TOP2 && (c->cap_b != 0 || c->E < 2)) return EC_ERR_INVALID_ARG;
+  if (D) { D->router = c->router; D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
            D->slots = (int64_t)c->E * D->k; D->d = c->d_model; D->dff = c->d_ff;
            D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb;
            D->cap_b = c->cap_b; D->cap_iters = c->cap_iters; D->cap_lambda = c->cap_lambda; }
   return EC_OK;
 }
 
-struct SavedLayout { size_t S, I, G, row_ptr, slots, X_in, Z, H, X_e, total; };
+struct SavedLayout { size_t S, I, G, row_ptr, slots, X_in, Z, H, X_e, load, requested, total; };
 // with_z = false: the layout of the same tensors without Z (forward-only calls keep them in the workspace)
 SavedLayout saved_layout(const Dims& D, bool with_z = true) {
   SavedLayout L; size_t o = 0;
@@ -60,6 +62,8 @@ SavedLayout saved_layout(const Dims& D, bool with_z = true) {
   L.Z = take(with_z ? (size_t)D.slots * D.dff * D.eb : 0);
   L.H = take((size_t)D.slots * D.dff * D.eb);
   L.X_e = take((size_t)D.slots * D.d * 4);          // fp32 on both paths
+  L.load = take(D.router ? (size_t)D.groups * D.E * 4 : 0);         // token-choice contrast only
+  L.requested = take(D.router ? (size_t)D.groups * D.E * 4 : 0);
   L.total = o;
   return L;
 }
@@ -74,7 +78,7 @@ int dwg_splits(const Dims& D) {
   return (int)(p < 1 ? 1 : (p > 32 ? 32 : p));
 }
 
-struct WsLayout { size_t status, topk, inverse, cap_A, capped, fwd_end, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
+struct WsLayout { size_t status, topk, inverse, cap_A, capped, choice, fwd_end, dX_e, dG, dZ, dX_in, dL, dWg_part, total; };
 WsLayout ws_layout(const Dims& D) {
   WsLayout L; size_t o = 0;
   auto take = [&](size_t b) { size_t r = o; o += up(b); return r; };
@@ -84,6 +88,7 @@ WsLayout ws_layout(const Dims& D) {
   L.inverse = take(inverse_scratch_bytes(D.n));
   L.cap_A = take(D.cap_b ? (size_t)D.n * D.E * 4 : 0);
   L.capped = take(D.cap_b ? capped_scratch_bytes(D.n, D.E, D.groups) : 0);
+  L.choice = take(D.router ? (size_t)D.n * 2 * 4 : 0);              // every token's two experts (token-choice contrast)
   const size_t fwd_end = o;
   L.fwd_end = fwd_end;
   o = base;                                   // the backward pass reuses the same region
@@ -140,6 +145,7 @@ struct BatchedGemm {
   int M, N, K, batches, epi;
   void* C2; const void* Zin;
   int c_f32;                                         // C is fp32 regardless of the path's dtype
+  const int32_t* batch_rows; int ragged;             // see TcGemmArgs: meaningful rows per batch along M (1) or K (2)
 };
 
 ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaStream_t st) {
@@ -150,6 +156,7 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
     t.lda = b.lda; t.ldb = b.ldb; t.batch_a = b.batch_a; t.batch_b = b.batch_b;
     t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c; t.c_f32 = b.c_f32;
     t.status = status_word;
+    t.batch_rows = b.batch_rows; t.ragged = b.ragged;
     if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); return EC_OK; }
   }
   GemmArgs g; memset(&g, 0, sizeof(g));
@@ -165,7 +172,8 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
 }
 
 ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int32_t* I, float* G,
-                     int32_t* row_ptr, int32_t* slots, char* ws, const WsLayout& W, cudaStream_t st) {
+                     int32_t* row_ptr, int32_t* slots, char* ws, const WsLayout& W, cudaStream_t st,
+                     int32_t* load = nullptr, int32_t* requested = nullptr) {
   bool done = false;
   if (D.dtype == EC_BF16) {
     TcGemmArgs t; memset(&t, 0, sizeof(t));
@@ -176,6 +184,15 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
   }
   if (!done) EC_CUDA(launch_gate_softmax_simt(D.dtype, X, Wg, S, D.n, D.d, D.E, st));
   prof_mark("gate_softmax", st);
+  if (D.router == EC_ROUTER_TOKEN_TOP2) {            // Section 3.1's token choice as a contrast: tokens pick, experts have buffers
+    int32_t* choice = (int32_t*)(ws + W.choice);
+    EC_CUDA(launch_token_top2(S, D.n, D.E, choice, st));
+    EC_CUDA(launch_token_admit(S, choice, D.ng, D.E, D.kg, D.groups, I, G, load, requested, st));
+    prof_mark("token_choice", st);
+    EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
+    prof_mark("inverse_index", st);
+    return EC_OK;
+  }
   const float* keys = S;
   if (D.cap_b) {                                    // Section 3.3: TopK(A, k) instead of TopK(S^T, k)
     float* A = (float*)(ws + W.cap_A);
@@ -254,12 +271,15 @@ ec_status ec_saved_view(const ec_config* c, void* saved, ec_saved_ptrs* out) {
   out->S = (float*)(b + L.S); out->I = (int32_t*)(b + L.I); out->G = (float*)(b + L.G);
   out->row_ptr = (int32_t*)(b + L.row_ptr); out->slots = (int32_t*)(b + L.slots);
   out->X_in = b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = (float*)(b + L.X_e);
+  out->load = D.router ? (int32_t*)(b + L.load) : nullptr;
+  out->requested = D.router ? (int32_t*)(b + L.requested) : nullptr;
   return EC_OK;
 }
 
 ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, int32_t* I, float* G,
                    int32_t* row_ptr, int32_t* slots, void* ws, size_t ws_bytes, void* stream) {
   Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (D.router != EC_ROUTER_EXPERT_CHOICE) return EC_ERR_INVALID_ARG;      // ec_route_token_choice has the outputs for that
   if (!X || !Wg || !S || !I || !G || !row_ptr || !slots || !ws) return EC_ERR_INVALID_ARG;
   if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(S, 16) || misaligned(I, 16) || misaligned(G, 16) ||
       misaligned(row_ptr, 16) || misaligned(slots, 16) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
@@ -269,6 +289,23 @@ ec_status ec_route(const ec_config* c, const void* X, const void* Wg, float* S, 
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   prof_begin(st, 0);
   return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st);
+}
+
+ec_status ec_route_token_choice(const ec_config* c, const void* X, const void* Wg, float* S, int32_t* I, float* G,
+                                int32_t* row_ptr, int32_t* slots, int32_t* load, int32_t* requested, void* ws,
+                                size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (D.router != EC_ROUTER_TOKEN_TOP2) return EC_ERR_INVALID_ARG;
+  if (!X || !Wg || !S || !I || !G || !row_ptr || !slots || !load || !requested || !ws) return EC_ERR_INVALID_ARG;
+  if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(S, 16) || misaligned(I, 16) || misaligned(G, 16) ||
+      misaligned(row_ptr, 16) || misaligned(slots, 16) || misaligned(load, 4) || misaligned(requested, 4) ||
+      misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D);
+  if (ws_bytes < W.total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  prof_begin(st, 0);
+  return route_impl(D, X, Wg, S, I, G, row_ptr, slots, (char*)ws, W, st, load, requested);
 }
 
 ec_status ec_capped_assignment(const ec_config* c, const float* S, float* A, void* ws, size_t ws_bytes, void* stream) {
@@ -318,6 +355,7 @@ size_t ec_route_static_bytes(const ec_config* c) {
 ec_status ec_route_static(const ec_config* c, const void* X, const void* Wg, float* S, int32_t* I, float* G,
                           int32_t* row_ptr, int32_t* slots, void* stream) {
   Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (D.router != EC_ROUTER_EXPERT_CHOICE) return EC_ERR_INVALID_ARG;
   if (!X || !Wg || !S || !I || !G || !row_ptr || !slots) return EC_ERR_INVALID_ARG;
   if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(S, 16) || misaligned(I, 16) || misaligned(G, 16) ||
       misaligned(row_ptr, 16) || misaligned(slots, 16)) return EC_ERR_INVALID_ARG;
@@ -351,16 +389,21 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   int* status = (int*)(w + W.status);
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   prof_begin(st, 0);
-  if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st)) != EC_OK) return s;
+  // token-choice contrast: slots filled per expert; with one routing group they are a prefix of the expert's buffer and
+  // the tensor-core GEMMs skip what lies beyond
+  int32_t* load = D.router ? (int32_t*)(sv + L.load) : nullptr;
+  int32_t* requested = D.router ? (int32_t*)(sv + L.requested) : nullptr;
+  const int32_t* rag = D.router && D.groups == 1 ? load : nullptr;
+  if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st, load, requested)) != EC_OK) return s;
   EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
   prof_mark("gather", st);
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Z = X_in[i] . W1[i],  H = GeLU(Z)
-  BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr};
+  BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr, 0, rag, 1};
   if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
   prof_mark("gemm1_gelu", st);
   // X_e = H[i] . W2[i]^T, kept in fp32
-  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1};
+  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1, rag, 1};
   if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
   prof_mark("gemm2", st);
   EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
@@ -387,6 +430,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   void* dX_e = w + W.dX_e; float* dG = (float*)(w + W.dG); void* dZ = w + W.dZ; void* dX_in = w + W.dX_in;
   void* dL = w + W.dL; float* part = (float*)(w + W.dWg_part);
   int* status = (int*)(w + W.status);
+  const int32_t* rag = D.router && D.groups == 1 ? (const int32_t*)(sv + L.load) : nullptr;   // see ec_moe_forward
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Eq. 4 backward: dX_e, dG
@@ -394,19 +438,19 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
   prof_mark("bwd_combine", st);
   // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
-  BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z};
+  BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z, 0, rag, 1};
   if ((s = run_gemm(D, g3, status, st)) != EC_OK) return s;
   prof_mark("gemm_dZ", st);
   // dW2[i] = dX_e[i]^T . H[i]
-  BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
+  BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2};
   if ((s = run_gemm(D, g4, status, st)) != EC_OK) return s;
   prof_mark("gemm_dW2", st);
   // dW1[i] = X_in[i]^T . dZ[i]
-  BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr};
+  BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2};
   if ((s = run_gemm(D, g5, status, st)) != EC_OK) return s;
   prof_mark("gemm_dW1", st);
   // dX_in[i] = dZ[i] . W1[i]^T
-  BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr};
+  BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 1};
   if ((s = run_gemm(D, g6, status, st)) != EC_OK) return s;
   prof_mark("gemm_dXin", st);
   // softmax backward: dL [n, E]; bf16 when the two gate-gradient products below run on tensor cores

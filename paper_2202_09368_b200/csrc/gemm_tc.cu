@@ -89,6 +89,7 @@ struct TcParams {
   int k_split;                                       // batches are cuts of one product along K
   int skip_c;                                        // EPI_GELU: only H = GeLU(acc) is stored, the accumulator itself is not
   const int32_t* row_ptr; const int32_t* slots; const bf16* rows; int64_t ld_rows;   // EPI_ADD_SLOTS
+  const int32_t* batch_rows; int ragged;             // meaningful rows per batch along M (1) or K (2), zeros beyond
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -273,6 +274,16 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
                     *reinterpret_cast<unsigned*>(&p2), *reinterpret_cast<unsigned*>(&p3));
 }
 
+// Ragged batches (token-choice routing leaves empty slots at the end of an expert's buffer): the k-blocks tile
+// (b, mt) runs, 0 if it is skipped.  All three roles of a CTA call this with the same arguments and so agree.
+__device__ __forceinline__ int tile_kblocks(const TcParams& p, int b, int mt, int tile_rows) {
+  if (p.batch_rows == nullptr) return p.kblocks;
+  const int rows = p.batch_rows[b];
+  if (p.ragged == 1) return (mt > 0 && mt * tile_rows >= rows) ? 0 : p.kblocks;   // a batch's first row tile always runs
+  const int kb = (rows + BK - 1) / BK;
+  return kb < 1 ? 1 : (kb < p.kblocks ? kb : p.kblocks);
+}
+
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
@@ -343,7 +354,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
         // B columns of this CTA: per 256-wide MMA the pair's two halves of kBHalf columns each, side by side
         const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * kBHalf;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        const int kblocks = tile_kblocks(p, b, mt, TM);
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1)) { gave_up = true; break; }
           const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
           const int k0 = kb * BK + (p.k_split ? b * p.K : 0);
@@ -398,12 +410,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t a_lbo = p.a_mn ? BK * 128 : 16, b_lbo = p.b_mn ? BK * 128 : 16;
       const uint32_t a_step = p.a_mn ? 2048 : 32, b_step = p.b_mn ? 2048 : 32;
       int stage = 0; uint32_t phase = 0; int it = 0;
-      for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step, ++it) {
+      for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step) {
+        const int kblocks = tile_kblocks(p, tile / (p.tiles_m * p.tiles_n),
+                                         p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m, TM);
+        if (kblocks == 0) continue;                  // a tile of empty slots: no accumulator is used
         const int buf = kOneAcc ? 0 : it & 1; const uint32_t use = (uint32_t)(kOneAcc ? it : it >> 1);
+        ++it;
         if (!mbar_wait(tempty0 + 8 * buf, (use & 1) ^ 1, abort_flag, p.status, 2)) { gave_up = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status, 3)) { gave_up = true; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
@@ -434,10 +450,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int it = 0;
     uint32_t nchunk = 0;                           // chunks this warp has stored so far: picks the staging buffer
     const uint32_t tempty_leader = CTAS == 2 ? map_to_cta(tempty0, 0) : tempty0;
-    for (int tile = first_tile; tile < p.total_tiles; tile += tile_step, ++it) {
+    for (int tile = first_tile; tile < p.total_tiles; tile += tile_step) {
       const int b = tile / (p.tiles_m * p.tiles_n);
-        const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
-        const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
+      const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
+      const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
+      if (tile_kblocks(p, b, mt, TM) == 0) continue; // a tile of empty slots: nothing was accumulated, nothing is stored
       const int buf = kOneAcc ? 0 : it & 1; const uint32_t use = (uint32_t)(kOneAcc ? it : it >> 1);
       const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
@@ -654,6 +671,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (lane == 0) {                             // one arrival per warp frees the accumulator
         if constexpr (CTAS == 2) mbar_arrive_cluster(tempty_leader + 8 * buf); else mbar_arrive(tempty0 + 8 * buf);
       }
+      ++it;                                        // tiles this CTA has worked on (skipped ones do not count)
     }
   }
 
@@ -788,6 +806,7 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
   if (g.epi == EPI_ADD_SLOTS && (g.batches != 1 || g.c_f32 || !g.row_ptr || !g.slots || !g.rows || g.ld_rows % 8 ||
                                  ((uintptr_t)g.rows & 15))) return false;
   if ((int64_t)g.lda * 2 >= ((int64_t)1 << 40) || (int64_t)g.ldb * 2 >= ((int64_t)1 << 40)) return false;
+  if (g.batch_rows && (g.k_split || (g.ragged != 1 && g.ragged != 2))) return false;
   return true;
 }
 
@@ -831,6 +850,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   // one time is whole rows of C rather than 512-byte pieces 2*N bytes apart, and they share the A tile.
   p.n_fast = (int64_t)g.M * g.N > ((int64_t)g.M + g.N) * g.K ? 1 : 0;
   p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows;
+  p.batch_rows = g.batch_rows; p.ragged = g.ragged;
   switch (g.epi) {
     case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
                                    : launch_bn<EPI_STORE>(bn, ctas, ta, tb, tc, tc2, p, st);

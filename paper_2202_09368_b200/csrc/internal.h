@@ -38,6 +38,12 @@ cudaError_t launch_gate_softmax_simt(int dtype, const void* X, const void* Wg, f
 size_t topk_scratch_bytes(int64_t n, int E, int64_t k, int groups);
 cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups, int32_t* I, float* G,
                         void* scratch, cudaStream_t st);
+// Token-choice contrast (Section 3.1): every token's two best experts (ties: lower expert) into choice [rows, 2];
+// then, per expert and group, the requests in token order fill a buffer of k slots: I (-1 = empty), G (0 = empty),
+// load and requested [groups, E].
+cudaError_t launch_token_top2(const float* S, int64_t rows, int E, int32_t* choice, cudaStream_t st);
+cudaError_t launch_token_admit(const float* S, const int32_t* choice, int64_t n, int E, int64_t k, int groups,
+                               int32_t* I, float* G, int32_t* load, int32_t* requested, cudaStream_t st);
 size_t inverse_scratch_bytes(int64_t n);
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t slots_total, int32_t* row_ptr,
                                  int32_t* slots, void* scratch, cudaStream_t st);
@@ -107,6 +113,11 @@ struct TcGemmArgs {
   // EPI_ADD_SLOTS (bf16 C, batches == 1): C[m, :] = acc[m, :] + sum over q in [row_ptr[m], row_ptr[m+1]) of
   // rows[slots[q], :] in ascending q, summed in fp32 and rounded once.
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;
+  // batch_rows != null: batch b holds only batch_rows[b] meaningful rows along its ragged dimension and zeros after
+  // them.  ragged = 1: that dimension is M; row tiles that start at or beyond batch_rows[b] are skipped (never the
+  // first one, so rows 0 .. tile-1 of C are always written).  ragged = 2: it is K; k-blocks that start at or beyond
+  // batch_rows[b] are skipped (at least one is run).
+  const int32_t* batch_rows; int ragged;
 };
 constexpr int EPI_SOFTMAX = 4;
 bool tc_gemm_supported(const TcGemmArgs& g);

@@ -710,6 +710,82 @@ cudaError_t launch_topk(const float* S, int64_t n, int E, int64_t k, int groups,
 }
 
 // ------------------------------------------------------------------------------------------
+// Token-choice contrast routing (Section 3.1): every token picks its two best experts, experts have buffers.
+// ------------------------------------------------------------------------------------------
+// One warp per token row of S: the two largest scores, equal scores to the lower expert.  A score in [0, 1] orders
+// like its bit pattern; the key puts the inverted expert index below it so that one max decides both.
+__global__ void __launch_bounds__(256) token_top2_kernel(const float* __restrict__ S, int64_t rows, int E, int32_t* __restrict__ choice) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < rows; t += warps) {
+    unsigned long long best = 0, second = 0;           // 0 is below every real key (the index part of a real key is > 0)
+    for (int i = lane; i < E; i += 32) {
+      const unsigned long long key = ((unsigned long long)__float_as_uint(S[t * E + i]) << 32) | (0xFFFFFFFFu - (unsigned)i);
+      if (key > best) { second = best; best = key; } else if (key > second) second = key;
+    }
+    unsigned long long top = best;
+    for (int o = 16; o; o >>= 1) { const unsigned long long v = __shfl_xor_sync(0xffffffffu, top, o); top = v > top ? v : top; }
+    const unsigned long long mine = best == top ? second : best;          // the winner's lane offers its runner-up
+    unsigned long long nxt = mine;
+    for (int o = 16; o; o >>= 1) { const unsigned long long v = __shfl_xor_sync(0xffffffffu, nxt, o); nxt = v > nxt ? v : nxt; }
+    if (lane == 0) {
+      choice[2 * t] = (int32_t)(0xFFFFFFFFu - (unsigned)top);
+      choice[2 * t + 1] = (int32_t)(0xFFFFFFFFu - (unsigned)nxt);
+    }
+  }
+}
+
+// One CTA per (expert, group) walks the group's tokens in order; a token that chose the expert takes the next slot
+// while there is one.  A token's two choices are different experts, so the order of the requests to one expert is
+// the token order.  Empty slots get -1 / 0.
+__global__ void __launch_bounds__(1024)
+token_admit_kernel(const float* __restrict__ S, const int32_t* __restrict__ choice, int n, int E, int k,
+                   int32_t* __restrict__ I, float* __restrict__ G, int32_t* __restrict__ load, int32_t* __restrict__ requested) {
+  __shared__ unsigned s_warp[33];
+  const int e = blockIdx.x, grp = blockIdx.y, groups = gridDim.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t row0 = (int64_t)grp * n;
+  int32_t* Ie = I + ((int64_t)e * groups + grp) * k;
+  float* Ge = G + ((int64_t)e * groups + grp) * k;
+  unsigned running = 0;
+  for (int base = 0; base < n; base += 1024) {
+    const int t = base + tid;
+    bool m = false;
+    if (t < n) { const int2 c = *reinterpret_cast<const int2*>(choice + 2 * (row0 + t)); m = c.x == e || c.y == e; }
+    const unsigned bal = __ballot_sync(0xffffffffu, m);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    if (warp == 0) {
+      const unsigned v = s_warp[lane];
+      unsigned inc = v;
+      for (int o = 1; o < 32; o <<= 1) { const unsigned u = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += u; }
+      s_warp[lane] = inc - v;
+      if (lane == 31) s_warp[32] = inc;
+    }
+    __syncthreads();
+    const unsigned pos = running + s_warp[warp] + __popc(bal & ((1u << lane) - 1u));
+    if (m && pos < (unsigned)k) { Ie[pos] = (int32_t)(row0 + t); Ge[pos] = S[(row0 + t) * E + e]; }
+    running += s_warp[32];
+    __syncthreads();
+  }
+  const unsigned filled = running < (unsigned)k ? running : (unsigned)k;
+  for (int j = (int)filled + tid; j < k; j += 1024) { Ie[j] = -1; Ge[j] = 0.f; }
+  if (tid == 0) { load[grp * E + e] = (int32_t)filled; requested[grp * E + e] = (int32_t)running; }
+}
+
+cudaError_t launch_token_top2(const float* S, int64_t rows, int E, int32_t* choice, cudaStream_t st) {
+  count_launch();
+  token_top2_kernel<<<grid_for(rows * 32, 256, 148 * 8), 256, 0, st>>>(S, rows, E, choice);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_token_admit(const float* S, const int32_t* choice, int64_t n, int E, int64_t k, int groups,
+                               int32_t* I, float* G, int32_t* load, int32_t* requested, cudaStream_t st) {
+  count_launch();
+  token_admit_kernel<<<dim3(E, groups), 1024, 0, st>>>(S, choice, (int)n, E, (int)k, I, G, load, requested);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
 // Index form of P = Onehot(I) (Eq. 2) read by token: row_ptr / slots.
 // Integer atomics only count and hand out positions; each token's short list is then sorted,
 // so the result does not depend on the order in which threads ran.
@@ -722,8 +798,10 @@ size_t inverse_scratch_bytes(int64_t n) {
 }
 
 __global__ void inv_count_kernel(const int32_t* __restrict__ I, int64_t total, int32_t* cnt) {
-  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x)
-    atomicAdd(&cnt[I[s]], 1);
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
+    const int t = I[s];
+    if (t >= 0) atomicAdd(&cnt[t], 1);                 // -1: an empty slot (token-choice routing only)
+  }
 }
 
 // Exclusive scan of the CTA's per-thread values (any thread count that is a multiple of 32, at most 1024);
@@ -780,7 +858,7 @@ __global__ void inv_fill_kernel(const int32_t* __restrict__ I, int64_t total, co
                                 int32_t* cnt, int32_t* slots) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
     const int t = I[s];
-    slots[row_ptr[t] + atomicSub(&cnt[t], 1) - 1] = (int32_t)s;
+    if (t >= 0) slots[row_ptr[t] + atomicSub(&cnt[t], 1) - 1] = (int32_t)s;
   }
 }
 
@@ -806,7 +884,7 @@ inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_p
   const int tid = threadIdx.x;
   for (int t = tid; t < n; t += 1024) s_cnt[t] = 0;
   __syncthreads();
-  for (int s = tid; s < total; s += 1024) atomicAdd(&s_cnt[I[s]], 1);
+  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0) atomicAdd(&s_cnt[t], 1); }
   __syncthreads();
   // exclusive scan over the tokens, 1024 * per at a time
   const int per = (n + 1023) / 1024, a = min(n, tid * per), b = min(n, a + per);
@@ -817,7 +895,7 @@ inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_p
   for (int t = a; t < b; ++t) { const int c = s_cnt[t]; row_ptr[t] = run; s_cnt[t] = run; run += c; }   // s_cnt becomes the cursor
   if (tid == 0) row_ptr[n] = total_sum;
   __syncthreads();
-  for (int s = tid; s < total; s += 1024) slots[atomicAdd(&s_cnt[I[s]], 1)] = s;
+  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0) slots[atomicAdd(&s_cnt[t], 1)] = s; }
   __syncthreads();
   __threadfence_block();
   for (int t = tid; t < n; t += 1024) {                // after the fill s_cnt[t] is the end of token t's list
@@ -845,7 +923,7 @@ inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row
   const int gtid = rank * 1024 + tid, gsize = nc * 1024;
   for (int t = gtid; t < n; t += gsize) cnt[t] = 0;
   inv_cluster_sync();
-  for (int s = gtid; s < total; s += gsize) atomicAdd(&cnt[I[s]], 1);
+  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0) atomicAdd(&cnt[t], 1); }
   inv_cluster_sync();
   // exclusive scan: CTA `rank` takes tokens [lo, hi), a thread `per` consecutive ones of them
   const int per_cta = (n + nc - 1) / nc, lo = min(n, rank * per_cta), hi = min(n, lo + per_cta);
@@ -867,7 +945,7 @@ inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row
   for (int t = a; t < b; ++t) { const int c = cnt[t]; row_ptr[t] = run; cnt[t] = run; run += c; }      // cnt becomes the cursor
   if (rank == nc - 1 && tid == 0) row_ptr[n] = before + tile;
   inv_cluster_sync();
-  for (int s = gtid; s < total; s += gsize) slots[atomicAdd(&cnt[I[s]], 1)] = s;
+  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0) slots[atomicAdd(&cnt[t], 1)] = s; }
   inv_cluster_sync();
   for (int t = gtid; t < n; t += gsize) {
     const int p0 = row_ptr[t], p1 = row_ptr[t + 1];
@@ -924,7 +1002,8 @@ __global__ void gather_kernel(const uint4* __restrict__ X, const int32_t* __rest
                               int64_t total_vec, int vec_per_row) {
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_vec; g += (int64_t)gridDim.x * blockDim.x) {
     const int64_t s = g / vec_per_row; const int v = (int)(g % vec_per_row);
-    X_in[g] = X[(int64_t)I[s] * vec_per_row + v];
+    const int t = I[s];                                // -1: an empty slot (token-choice routing only) holds a zero row
+    X_in[g] = t >= 0 ? X[(int64_t)t * vec_per_row + v] : make_uint4(0, 0, 0, 0);
   }
 }
 
@@ -1010,6 +1089,12 @@ __global__ void bwd_combine_kernel(const T* __restrict__ dX_out, const float* __
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t s = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; s < total; s += warps) {
     const int64_t t = I[s];
+    if (t < 0) {                                       // an empty slot (token-choice routing only): zero row, no gradient
+      const float z[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int v = lane; v < quads_per_row; v += 32) store4(dX_e + (s * quads_per_row + v) * 4, z);
+      if (lane == 0) dG[s] = 0.f;
+      continue;
+    }
     const float w = G[s];
     float dot = 0.f;
     for (int v = lane; v < quads_per_row; v += 32) {

@@ -76,10 +76,19 @@ class LayerInputs:
 
 
 def make_layer_inputs(n: int, d: int, dff: int, E: int, dtype=torch.float32, seed: int = 0,
-                      logit_scale: float = 1.0, device="cpu", with_grad: bool = True) -> LayerInputs:
-    """Inputs of one layer call.  `logit_scale` multiplies Wg (varies the token-score skew)."""
+                      logit_scale: float = 1.0, device="cpu", with_grad: bool = True,
+                      expert_skew: float = 0.0) -> LayerInputs:
+    """Inputs of one layer call.  `logit_scale` multiplies Wg (varies the token-score skew).
+
+    `expert_skew` > 0 makes some experts popular with every token, the way a trained gate without a balancing
+    loss does: feature 0 of every token is set to 1 and row 0 of Wg to expert_skew * z_i with z ~ N(0, 1), which
+    adds the same logit offset z_i * expert_skew to expert i for all tokens (the layer has no bias term to carry it).
+    """
     X = normal_tensor((n, d), 1.0, seed, TID_X, dtype, device)
     Wg = normal_tensor((d, E), logit_scale / math.sqrt(d), seed, TID_WG, dtype, device)
+    if expert_skew:
+        X[:, 0] = 1.0
+        Wg[0, :] = (normal_chunk(seed, TID_AUX, 1 << 20, E, device) * expert_skew).to(dtype)
     W1 = normal_tensor((E, d, dff), 1.0 / math.sqrt(d), seed, TID_W1, dtype, device)
     W2 = normal_tensor((E, d, dff), 1.0 / math.sqrt(dff), seed, TID_W2, dtype, device)
     dX_out = normal_tensor((n, d), 1.0, seed, TID_DXOUT, dtype, device) if with_grad else None

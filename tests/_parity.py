@@ -71,6 +71,24 @@ def to_np(t):
 CAP_ATOL = 2e-3      # on entries of A in [0, 1]: fp32 rounding of log A (|log A| up to 1/lambda) carried through the rounds
 
 
+def check_token_choice(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots, load, requested):
+    """Step (ii) for the token-choice contrast: the oracle's walk over the GPU's own S must give the same slots,
+    gate weights, loads and request counts, and the same token -> slot index over the filled slots."""
+    k, n, g = B.ec_capacity(cfg), cfg.n, cfg.groups
+    S32 = S_gpu.cpu().numpy()
+    parts = [O.token_choice(S32[r * n:(r + 1) * n], k) for r in range(g)]
+    I_ref = np.concatenate([np.where(p[1] >= 0, p[1] + r * n, -1) for r, p in enumerate(parts)], axis=1)
+    G_ref = np.concatenate([p[0] for p in parts], axis=1)
+    assert np.array_equal(I_gpu.cpu().numpy(), I_ref), f"I differs in {(I_gpu.cpu().numpy() != I_ref).sum()} slots"
+    assert np.array_equal(G_gpu.cpu().numpy().view(np.uint32), G_ref.astype(np.float32).view(np.uint32))
+    assert np.array_equal(load.cpu().numpy(), np.stack([p[2] for p in parts]))
+    assert np.array_equal(requested.cpu().numpy(), np.stack([p[3] for p in parts]))
+    rp_ref, sl_ref = O.inverse_index(I_ref, n * g)
+    assert np.array_equal(row_ptr.cpu().numpy(), rp_ref)
+    assert np.array_equal(slots.cpu().numpy()[:len(sl_ref)], sl_ref)
+    return I_ref
+
+
 def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
     """Step (ii): bit-exact routing given the GPU's own S.  With a cap (Section 3.3) the GPU's A is compared with
     the oracle's by tolerance and the indices must be the oracle's TopK of the GPU's own A, the gate weights S at them."""
@@ -97,11 +115,11 @@ def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
     return I_ref
 
 
-def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1, **cap):
+def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1, router="expert", **cap):
     """Runs forward (+ backward) on the GPU and checks every tensor against the oracle.
     n is the number of tokens per routing group; li holds groups * n rows."""
     tol = TOL[dtype]
-    cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups, **cap)
+    cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups, router=router, **cap)
     dev = "cuda"
     X, Wg, W1, W2 = (t.to(dev) for t in (li.X, li.Wg, li.W1, li.W2))
     ws = B.alloc_workspace(cfg)
@@ -113,12 +131,21 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
     if check_S:
         errs["S"] = rel_err(to_np(v["S"]), O.gate(Xn, Wgn))
         assert errs["S"] <= tol, errs
-    check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
-    f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(), groups=groups)
-    assert np.array_equal(v["X_in"].float().cpu().numpy(), Xn[f["I"]].astype(np.float32))   # the shuffle of Eq. 3 is a copy
+    if router == "token":
+        check_token_choice(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"], v["load"], v["requested"])
+    else:
+        check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
+    f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(), groups=groups,
+                  router=router)
+    assert np.array_equal(v["X_in"].float().cpu().numpy(), f["X_in"].astype(np.float32))    # the shuffle of Eq. 3 is a copy
+    filled = v["I"].cpu().numpy() >= 0             # all slots with expert choice; token choice leaves some empty, and
+    got = {}                                       # what the library keeps for an empty slot is unspecified
     for name in ("Z", "H", "X_e"):
-        errs[name] = rel_err(to_np(v[name]), f[name])
-    errs["X_out"] = rel_err(to_np(X_out), f["X_out"])
+        got[name] = to_np(v[name])
+        got[name][~filled] = 0.0
+        errs[name] = rel_err(got[name], f[name])
+    got["X_out"] = to_np(X_out)
+    errs["X_out"] = rel_err(got["X_out"], f["X_out"])
     cnt = O.experts_per_token(f["row_ptr"])
     assert torch.all(X_out[torch.from_numpy(cnt == 0).to(dev)] == 0)
     if backward:
@@ -127,24 +154,23 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         assert B.ec_read_status(ws) == B.EC_OK
         b = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), f, gelu)
         for name, t in (("dX", dX), ("dWg", dWg), ("dW1", dW1), ("dW2", dW2)):
-            errs[name] = rel_err(to_np(t), b[name])
+            got[name] = to_np(t)
+            errs[name] = rel_err(got[name], b[name])
     bound = {k_: tol for k_ in errs}
     bad = {k_: (e, bound[k_]) for k_, e in errs.items() if not e <= bound[k_]}
     if dtype == torch.bfloat16:
         rec = Bf16Recorder()
         ff = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(),
-                       store=rec, groups=groups)
-        got = {"Z": v["Z"], "H": v["H"], "X_e": v["X_e"], "X_out": X_out}
+                       store=rec, groups=groups, router=router)
         refs = dict(f)
         if backward:
             fb = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), ff, gelu, store=rec)
-            got.update(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2)
             refs.update(b)
             ff = {**ff, **fb}
         detail, bad = {}, {k_: v_ for k_, v_ in bad.items() if k_ == "S"}
         for k_, t in got.items():
             stored = k_ in BF16_STORED
-            a = bf16_assess(to_np(t), refs[k_], rec.before(k_, refs[k_]) if stored else ff[k_], stored, k_)
+            a = bf16_assess(t, refs[k_], rec.before(k_, refs[k_]) if stored else ff[k_], stored, k_)
             detail[k_] = a
             if not a["ok"]:
                 bad[k_] = a
