@@ -565,6 +565,51 @@ def run_sweep(args):
                       "cases": cases}))
 
 
+# ----------------------------------------------------------------------------------- expert GEMMs alone
+def run_gemms(args):
+    """The three expert-batched products of the layer, each alone in a loop (ec_expert_gemm), and torch.bmm (the vendor
+    library) on the same buffers beside them, alternating, for calibration: what the tensor cores give this shape when
+    nothing else runs.  16 experts of the workload's shape (the weight gradients then write 2 GiB per call at 8B/64E)."""
+    import torch
+    from paper_2202_09368_b200 import binding as B
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    dev, bf = torch.device("cuda"), torch.bfloat16
+    n, d, dff, E, c = WORKLOADS[args.workload]
+    Eb = min(E, 16)
+    cfg = B.make_config(n * Eb // E, d, dff, Eb, c, bf)
+    k = B.ec_capacity(cfg)
+    A = torch.randn(Eb, k, d, device=dev, dtype=bf)
+    H = torch.randn(Eb, k, dff, device=dev, dtype=bf)
+    W = torch.randn(Eb, d, dff, device=dev, dtype=bf) * 0.02
+    ws = B.alloc_workspace(cfg, dev)
+    outs = {B.EC_GEMM_XW1: torch.empty(Eb, k, dff, device=dev, dtype=bf), B.EC_GEMM_HW2T: torch.empty(Eb, k, d, device=dev, dtype=bf),
+            B.EC_GEMM_ATB: torch.empty(Eb, d, dff, device=dev, dtype=bf)}
+    flops = 2.0 * Eb * k * d * dff
+    cases = [("Z = X_in . W1", B.EC_GEMM_XW1, A, W, lambda o: torch.bmm(A, W, out=o)),
+             ("X_e = H . W2^T", B.EC_GEMM_HW2T, H, W, lambda o: torch.bmm(H, W.transpose(1, 2), out=o)),
+             ("dW = A^T . B", B.EC_GEMM_ATB, A, H, lambda o: torch.bmm(A.transpose(1, 2), H, out=o))]
+    reps = max(10, args.steps)
+    res = {}
+    for rnd in range(max(2, min(args.repeats, 3))):
+        for name, kind, a, b_, vendor in cases:
+            o = outs[kind]
+            for tag, fn in (("this_library", lambda: B.ec_expert_gemm(cfg, kind, a, b_, o, ws)), ("torch_bmm", lambda: vendor(o))):
+                for _ in range(5):
+                    fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(reps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                res.setdefault(name, {}).setdefault(tag, []).append(round(flops / (e0.elapsed_time(e1) / reps) / 1e9, 1))
+    assert B.ec_read_status(ws) == B.EC_OK
+    print(json.dumps({"metric": "expert_gemm_alone_tflops", "unit": "TFLOP/s, each product alone in a loop, rounds in order",
+                      "config": {"workload": f"{Eb} experts of {args.workload}: k={k} d={d} d_ff={dff}, bf16", "calls_per_timing": reps},
+                      "cases": res}))
+
+
 # ----------------------------------------------------------------------------------- token-choice contrast
 def run_contrast(args):
     """Expert choice next to the token-choice top-2 routing it is contrasted with (Section 3.1, Section 4.2), on
@@ -655,10 +700,13 @@ def main():
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")
+    ap.add_argument("--gemms", action="store_true", help="the expert GEMMs alone in a loop, torch.bmm beside them (calibration)")
     ap.add_argument("--contrast", action="store_true", help="expert choice beside token-choice top-2 routing on identical inputs")
     ap.add_argument("--expert-skew", type=float, default=0.05, help="with --contrast: popularity offset of the experts' gate logits")
     args = ap.parse_args()
-    if args.contrast:
+    if args.gemms:
+        run_gemms(args)
+    elif args.contrast:
         run_contrast(args)
     elif args.sweep:
         run_sweep(args)

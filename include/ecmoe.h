@@ -247,6 +247,19 @@ ec_status ec_moe_backward(const ec_config* cfg, const void* X, const void* Wg, c
                           size_t ws_bytes, void* cuda_stream);
 
 /*
+ * One expert-batched product of Eq. 3 or of its backward on its own (benchmarks time the kernels apart from the layer
+ * with it; ec_moe_forward / ec_moe_backward run the same kernels).  k = ec_capacity(cfg) * groups rows per expert,
+ * d = d_model, d' = d_ff, all operands and the result of cfg->dtype, dense, [E, rows, columns]:
+ *   EC_GEMM_XW1   C[i] = A[i] . B[i]        A [E, k, d],  B [E, d, d'] (W1's layout)       -> C [E, k, d']
+ *   EC_GEMM_HW2T  C[i] = A[i] . B[i]^T      A [E, k, d'], B [E, d, d'] (W2's layout)       -> C [E, k, d]
+ *   EC_GEMM_ATB   C[i] = A[i]^T . B[i]      A [E, k, d],  B [E, k, d'] (the weight gradients) -> C [E, d, d']
+ * fp32 accumulation, one rounding to cfg->dtype.  `ws` as for the other calls (only its status word is used).
+ */
+typedef enum { EC_GEMM_XW1 = 0, EC_GEMM_HW2T = 1, EC_GEMM_ATB = 2 } ec_gemm_kind;
+ec_status ec_expert_gemm(const ec_config* cfg, int kind, const void* A, const void* B, void* C, void* ws,
+                         size_t ws_bytes, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and reads the status word the kernels of the last call
  * on `ws` left there: EC_OK, or EC_ERR_TIMEOUT when a bounded wait inside a kernel
  * gave up (the outputs of that call are then undefined), or EC_ERR_CUDA when the

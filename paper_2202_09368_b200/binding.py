@@ -24,7 +24,8 @@ EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
            "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
-           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice"]
+           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice", "ec_expert_gemm"]
+EC_GEMM_XW1, EC_GEMM_HW2T, EC_GEMM_ATB = 0, 1, 2
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -64,6 +65,8 @@ def lib():
         L.ec_route.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V]
         L.ec_route_token_choice.restype = C.c_int
         L.ec_route_token_choice.argtypes = [P, V, V, V, V, V, V, V, V, V, V, C.c_size_t, V]
+        L.ec_expert_gemm.restype = C.c_int
+        L.ec_expert_gemm.argtypes = [P, C.c_int, V, V, V, V, C.c_size_t, V]
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
@@ -228,6 +231,17 @@ def ec_unshuffle(cfg, X_e, G, row_ptr, slots, X_out=None):
     _check(lib().ec_unshuffle(C.byref(cfg), _ptr(X_e), _ptr(G), _ptr(row_ptr), _ptr(slots), _ptr(X_out), _stream()),
            "ec_unshuffle")
     return X_out
+
+
+def ec_expert_gemm(cfg, kind, A, Bm, out=None, ws=None):
+    """One expert-batched product of Eq. 3 / its backward on its own (see ecmoe.h for the three kinds and shapes)."""
+    k, E, d, f = slots_per_expert(cfg), cfg.E, cfg.d_model, cfg.d_ff
+    shape = {EC_GEMM_XW1: (E, k, f), EC_GEMM_HW2T: (E, k, d), EC_GEMM_ATB: (E, d, f)}[kind]
+    out = torch.empty(shape, dtype=A.dtype, device=A.device) if out is None else out
+    ws = alloc_workspace(cfg, A.device) if ws is None else ws
+    _check(lib().ec_expert_gemm(C.byref(cfg), kind, _ptr(A), _ptr(Bm), _ptr(out), _ptr(ws), ws.numel(), _stream()),
+           "ec_expert_gemm")
+    return out
 
 
 def ec_route_static_bytes(cfg: ec_config) -> int:

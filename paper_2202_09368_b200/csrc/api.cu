@@ -502,6 +502,26 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   return EC_OK;
 }
 
+ec_status ec_expert_gemm(const ec_config* c, int kind, const void* A, const void* B, void* C, void* ws, size_t ws_bytes,
+                         void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (kind != EC_GEMM_XW1 && kind != EC_GEMM_HW2T && kind != EC_GEMM_ATB) return EC_ERR_INVALID_ARG;
+  if (!A || !B || !C || !ws || misaligned(A, 16) || misaligned(B, 16) || misaligned(C, 16) || misaligned(ws, kAlign))
+    return EC_ERR_INVALID_ARG;
+  if (ws_bytes < ws_layout(D).total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
+  const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
+  BatchedGemm g;
+  if (kind == EC_GEMM_XW1) g = {A, 0, D.d, kd, B, 1, D.dff, df, C, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
+  else if (kind == EC_GEMM_HW2T) g = {A, 0, D.dff, kf, B, 0, D.dff, df, C, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
+  else g = {A, 1, D.d, kd, B, 1, D.dff, kf, C, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
+  prof_begin(st, 0);
+  s = run_gemm(D, g, (int*)ws, st);
+  prof_mark("expert_gemm", st);
+  return s;
+}
+
 ec_status ec_read_status(const void* ws, void* stream) {
   if (!ws) return EC_ERR_INVALID_ARG;
   StatusWord h;

@@ -147,6 +147,14 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
   asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// Named barriers over the four epilogue warps that share a half of the tile's columns (ids 1 and 2; 0 is __syncthreads).
+__device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, 128;" ::"r"(1 + half) : "memory"); }
+__device__ __forceinline__ bool half_all(int half, bool ok) {          // true when `ok` holds in all 128 threads
+  uint32_t r;
+  asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %2, 0;\n barrier.cta.red.and.pred q, %1, 128, p;\n selp.u32 %0, 1, 0, q;\n}\n"
+               : "=r"(r) : "r"(1 + half), "r"((uint32_t)ok) : "memory");
+  return r != 0;
+}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -457,7 +465,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (tile_kblocks(p, b, mt, TM) == 0) continue; // a tile of empty slots: nothing was accumulated, nothing is stored
       const int buf = kOneAcc ? 0 : it & 1; const uint32_t use = (uint32_t)(kOneAcc ? it : it >> 1);
       const bool ok = mbar_wait(tfull0 + 8 * buf, use & 1, abort_flag, p.status, 4);
-      if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
+      if constexpr (EPI == EPI_STORE) {
+        // the four warps of a column half meet at named barriers below: they leave together or not at all (every one
+        // of them gets here, its wait being bounded)
+        if (!half_all(half, ok)) { gave_up = true; break; }
+      } else {
+        if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
+      }
       tc_fence_after();
       const int row = mt * TM + (int)rank * BM + q * 32 + lane;
       const bool row_ok = row < p.M;
@@ -649,19 +663,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   }
                 }
               }
-              uint8_t* bufp = stg + (nchunk & 1) * 4096;
-              if (lane == 0) bulk_wait_read<1>();  // the other buffer's store may still be in flight
-              __syncwarp();
+              if constexpr (EPI == EPI_STORE) {
+                // Plain results leave in boxes of 128 rows: the four warps of this column half fill one 16 KiB buffer
+                // (two per half, alternating), one thread stores it.  Four stores per 128 x 256 block instead of sixteen:
+                // the weight gradients, which write a tile's 64 KiB per eight k-blocks, gain 3 % (8 % alone in a loop).
+                uint8_t* hb = smem + S * kStage + half * (4 * kStagingPerWarp) + (nchunk & 1) * 16384;
+                const bool leader = q == 0 && lane == 0;
+                if (leader) bulk_wait_read<1>();     // the store that last read this buffer (two chunks ago) is through with it
+                half_sync(half);
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float f[8];
+                for (int j = 0; j < 8; ++j) {
+                  float f[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * j + e]);
-                *reinterpret_cast<uint4*>(bufp + lane * 128 + ((j ^ sw) << 4)) = pack8(f);
+                  for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * j + e]);
+                  *reinterpret_cast<uint4*>(hb + (q * 32 + lane) * 128 + ((j ^ sw) << 4)) = pack8(f);
+                }
+                fence_async_smem();
+                half_sync(half);
+                const int rt0 = mt * TM + (int)rank * BM;
+                if (leader && rt0 < p.M) { tma_store_3d(&tmC, smem_u32(hb), n0 + c0, rt0, b); bulk_commit(); }
+              } else {
+                uint8_t* bufp = stg + (nchunk & 1) * 4096;
+                if (lane == 0) bulk_wait_read<1>();  // the other buffer's store may still be in flight
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  float f[8];
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(r[8 * j + e]);
+                  *reinterpret_cast<uint4*>(bufp + lane * 128 + ((j ^ sw) << 4)) = pack8(f);
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + (nchunk & 1) * 4096, n0 + c0, r0, b); bulk_commit(); }
               }
-              fence_async_smem();
-              __syncwarp();
-              if (lane == 0 && r0 < p.M) { tma_store_3d(&tmC, stg_s + (nchunk & 1) * 4096, n0 + c0, r0, b); bulk_commit(); }
             }
           }
         }
@@ -833,7 +868,9 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
     if (!make_map(&tc, g.S, g.N, g.M, 1, g.ldc, 0, 32, 32, true)) return cudaErrorInvalidValue;
   } else {
     const void* cbase = (g.epi == EPI_GELU && !g.C) ? g.C2 : g.C;     // without C its map is never used: any valid one will do
-    if (!make_map(&tc, cbase, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, 32, g.c_f32 != 0)) return cudaErrorInvalidValue;
+    // plain bf16 results are stored in boxes of 128 rows (a column half's four warps together), the rest in boxes of 32
+    if (!make_map(&tc, cbase, g.N, g.M, g.batches, g.ldc, g.batch_c, g.c_f32 ? 32 : 64, (g.epi == EPI_STORE && !g.c_f32) ? 128 : 32,
+                  g.c_f32 != 0)) return cudaErrorInvalidValue;
     if (g.epi == EPI_GELU && !make_map(&tc2, g.C2, g.N, g.M, g.batches, g.ldc, g.batch_c, 64, 32)) return cudaErrorInvalidValue;
   }
   TcParams p;

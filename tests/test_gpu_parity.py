@@ -100,6 +100,26 @@ def test_gate_with_more_experts_than_one_column_tile_and_few_rows(n, E, groups):
     check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
 
 
+@pytest.mark.parametrize("dtype,n,d,dff,E", [(F32, 200, 24, 40, 4), (BF16, 1024, 128, 384, 4), (BF16, 2048, 256, 2304, 4)])
+def test_expert_gemm_on_its_own(dtype, n, d, dff, E):
+    """The three expert-batched products of Eq. 3 and its backward as calls of their own, against numpy in fp64."""
+    cfg = B.make_config(n, d, dff, E, 2.0, dtype)
+    k = B.ec_capacity(cfg)
+    li = IN.make_layer_inputs(n, d, dff, E, dtype, seed=23)
+    A = li.X[:E * k // 2].repeat(2, 1).view(E, k, d).contiguous().cuda()                  # [E, k, d]
+    H = IN.normal_tensor((E, k, dff), 1.0, 23, IN.TID_AUX, dtype).cuda()                   # [E, k, d']
+    W1, W2 = li.W1.cuda(), li.W2.cuda()
+    tol = TOL[dtype]
+    for kind, a, b_, ref in ((B.EC_GEMM_XW1, A, W1, np.einsum("ikd,idf->ikf", to_np(A), to_np(W1))),
+                             (B.EC_GEMM_HW2T, H, W2, np.einsum("ikf,idf->ikd", to_np(H), to_np(W2))),
+                             (B.EC_GEMM_ATB, A, H, np.einsum("ikd,ikf->idf", to_np(A), to_np(H)))):
+        got = to_np(B.ec_expert_gemm(cfg, kind, a, b_))
+        if dtype == BF16:                      # one rounding of the exact result to bf16
+            assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-5 * np.sqrt(np.mean(ref ** 2))), kind
+        else:
+            assert rel_err(got, ref) <= tol, kind
+
+
 def test_read_status_maps_the_status_word():
     """ec_read_status only reads the first word of the workspace: 0 is EC_OK, 5 a bounded wait that expired, anything
     else is reported as a CUDA error.  No kernel is involved."""
