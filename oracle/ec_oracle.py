@@ -116,15 +116,22 @@ def gelu_grad(z, variant: str = "erf"):
     raise ValueError(variant)
 
 
-def expert_ffn(X_in_i, W1_i, W2_i, gelu_variant: str = "erf", store=_keep):
+def expert_ffn(X_in_i, W1_i, W2_i, gelu_variant: str = "erf", store=_keep, b1_i=None, b2_i=None):
     """Eq. 3 for one expert: Z = X_in[i] . W1[i], H = GeLU(Z), X_e[i] = H . W2[i]^T.
+    The paper leaves the bias terms out of Eq. 3 "for brevity"; given b1[i] (d') and b2[i] (d) they are the usual ones
+    of a feed-forward block, Z = X_in[i] . W1[i] + b1[i] and X_e[i] = H . W2[i]^T + b2[i].
 
     `store` (see forward()) is handed every tensor this function produces.  H is GeLU of the product
     itself, as Eq. 3 writes it, not of what `store` made of Z."""
     Z = X_in_i @ W1_i                                      # [k, d']
+    if b1_i is not None:
+        Z = Z + np.asarray(b1_i, F64)[None, :]
     H = store("H", gelu(Z, gelu_variant))
     Z = store("Z", Z)
-    X_e = store("X_e", H @ W2_i.T)                         # [k, d]
+    X_e = H @ W2_i.T                                       # [k, d]
+    if b2_i is not None:
+        X_e = X_e + np.asarray(b2_i, F64)[None, :]
+    X_e = store("X_e", X_e)
     return Z, H, X_e
 
 
@@ -274,12 +281,15 @@ def route(X, Wg, c: float, S_override=None, groups: int = 1, cap_b: int = 0, cap
 
 def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None, I_override=None,
             store=_keep, groups: int = 1, cap_b: int = 0, cap_lambda: float = 1e-3, cap_iters: int = 100,
-            router: str = "expert"):
+            router: str = "expert", b1=None, b2=None):
     """Eq. 1-4.  Returns every intermediate.
 
     S_override replaces the gate output (the routing is then taken from it);
     I_override additionally fixes the index matrix (G is read from S at I).
     Both exist so that later stages can be compared on identical routing.
+
+    b1 [e, d'] and b2 [e, d] are the bias terms Eq. 3 omits (see expert_ffn); None = the equation as printed.
+    With biases an empty slot (token choice only) no longer holds zeros in Z, H, X_e, but nothing reads them there.
 
     cap_b > 0 routes with the capped assignment of Section 3.3, router = "token" with the token-choice
     contrast of Section 3.1 (see route()); empty slots then hold zero rows throughout.
@@ -308,7 +318,8 @@ def forward(X, Wg, W1, W2, c: float, gelu_variant: str = "erf", S_override=None,
     if (I < 0).any():
         X_in[I < 0] = 0.0                                  # an empty slot (token choice only) holds a zero row
     X_in = store("X_in", X_in)
-    per_expert = [expert_ffn(X_in[i], W1[i], W2[i], gelu_variant, store) for i in range(e)]
+    per_expert = [expert_ffn(X_in[i], W1[i], W2[i], gelu_variant, store,
+                             None if b1 is None else b1[i], None if b2 is None else b2[i]) for i in range(e)]
     Z = np.stack([p[0] for p in per_expert])               # [e, k, d']
     H = np.stack([p[1] for p in per_expert])               # [e, k, d']
     X_e = np.stack([p[2] for p in per_expert])             # [e, k, d]
@@ -340,10 +351,13 @@ def backward(X, Wg, W1, W2, dX_out, fwd, gelu_variant: str = "erf", store=_keep)
     dX_in = np.stack([p[2] for p in per_expert])           # [e, k, d]
     dH = np.stack([p[3] for p in per_expert])
     dZ = np.stack([p[4] for p in per_expert])
+    filled = (I >= 0)[:, :, None]                          # gradients of the bias terms Eq. 3 omits: sums over an expert's filled slots
+    db1 = store("db1", (dZ * filled).sum(axis=1))          # [e, d']
+    db2 = store("db2", (dX_e * filled).sum(axis=1))        # [e, d]
     dS, dL = softmax_backward(S, I, dG, store)
     dWg = store("dWg", X.T @ dL)
     dX = store("dX", add_slot_rows(dL @ Wg.T, I, dX_in))
-    return dict(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2, dX_e=dX_e, dG=dG, dH=dH, dZ=dZ,
+    return dict(dX=dX, dWg=dWg, dW1=dW1, dW2=dW2, db1=db1, db2=db2, dX_e=dX_e, dG=dG, dH=dH, dZ=dZ,
                 dX_in=dX_in, dS=dS, dL=dL)
 
 

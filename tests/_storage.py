@@ -6,7 +6,7 @@ rounding it changes nothing; S, G, X_e, dG, dS, dH are fp32 or never stored on t
 """
 import numpy as np
 
-BF16_STORED = frozenset({"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2"})
+BF16_STORED = frozenset({"Z", "H", "X_out", "dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2", "db1", "db2"})
 
 
 def round_bf16(x):

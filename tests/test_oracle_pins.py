@@ -302,3 +302,52 @@ def test_routing_groups_are_independent_layers_on_the_blocks(groups, n, E, c):
         fd = (loss(*plus) - loss(*minus)) / (2 * h)
         an = float((b[name] * D).sum())
         assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (name, fd, an)
+
+
+# ---------------------------------------------------------------- the bias terms Eq. 3 omits
+def test_biases_dense_closed_form_and_zero_bias_is_no_bias():
+    """One expert that takes every token: the layer is a dense feed-forward block with biases, S = 1."""
+    n, d, dff = 40, 6, 10
+    X, Wg, W1, W2, dY = mk(n, d, dff, 1, seed=4)
+    rng = np.random.default_rng(2)
+    b1, b2 = rng.standard_normal((1, dff)), rng.standard_normal((1, d))
+    f = O.forward(X, Wg, W1, W2, 1.0, b1=b1, b2=b2)
+    z = X @ W1[0] + b1[0]
+    want = (z * 0.5 * (1 + np.vectorize(math.erf)(z / math.sqrt(2)))) @ W2[0].T + b2[0]
+    order = f["I"][0]
+    np.testing.assert_allclose(f["X_out"], want, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(f["Z"][0], z[order], rtol=1e-13, atol=1e-14)
+    # gradients of the dense block, written out independently
+    b = O.backward(X, Wg, W1, W2, dY, f)
+    Phi = 0.5 * (1 + np.vectorize(math.erf)(z / math.sqrt(2)))
+    dz = (dY @ W2[0]) * (Phi + z * np.exp(-0.5 * z * z) / math.sqrt(2 * math.pi))
+    np.testing.assert_allclose(b["db2"][0], dY.sum(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(b["db1"][0], dz.sum(axis=0), rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(b["dW1"][0], X.T @ dz, rtol=1e-11, atol=1e-13)
+    # zero biases change nothing, bit for bit
+    X, Wg, W1, W2, dY = mk(64, 8, 12, 4, seed=6)
+    f0 = O.forward(X, Wg, W1, W2, 2.0)
+    fz = O.forward(X, Wg, W1, W2, 2.0, b1=np.zeros((4, 12)), b2=np.zeros((4, 8)))
+    assert np.array_equal(f0["X_out"], fz["X_out"]) and np.array_equal(f0["Z"], fz["Z"])
+
+
+@pytest.mark.parametrize("router", ["expert", "token"])
+def test_bias_gradients_match_finite_differences(router):
+    n, d, dff, E, c = 40, 6, 10, 4, 1.9
+    X, Wg, W1, W2, dY = mk(n, d, dff, E, seed=13)
+    rng = np.random.default_rng(5)
+    b1, b2 = 0.5 * rng.standard_normal((E, dff)), 0.5 * rng.standard_normal((E, d))
+    f = O.forward(X, Wg, W1, W2, c, router=router, b1=b1, b2=b2)
+    b = O.backward(X, Wg, W1, W2, dY, f)
+    h = 1e-6
+    for name, key in (("db1", "b1"), ("db2", "b2"), ("dW1", "W1"), ("dX", "X")):
+        base = dict(X=X, W1=W1, b1=b1, b2=b2)
+        D = rng.standard_normal(base[key].shape)
+        vals = []
+        for sgn in (+1, -1):
+            a = dict(base); a[key] = base[key] + sgn * h * D
+            g = O.forward(a["X"], Wg, a["W1"], W2, c, router=router, b1=a["b1"], b2=a["b2"])
+            assert np.array_equal(g["I"], f["I"])
+            vals.append(float((dY * g["X_out"]).sum()))
+        fd, an = (vals[0] - vals[1]) / (2 * h), float((b[name] * D).sum())
+        assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (name, fd, an)

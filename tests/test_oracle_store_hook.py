@@ -53,7 +53,7 @@ def test_identity_hook_is_the_definition_and_sees_every_tensor_once():
             assert np.array_equal(np.asarray(a[k_]), np.asarray(b[k_])), k_
     per_expert_f, per_expert_b = ["H", "Z", "X_e"], ["dW2", "dZ", "dW1", "dX_in", "dH"]
     assert fwd_seen == ["X_in"] + per_expert_f * E + ["X_out"]
-    assert seen == ["dX_e", "dG"] + per_expert_b * E + ["dS", "dL", "dWg", "dX"]
+    assert seen == ["dX_e", "dG"] + per_expert_b * E + ["db1", "db2", "dS", "dL", "dWg", "dX"]
     assert BF16_STORED <= set(fwd_seen) | set(seen)          # every name the tests round is one the hook is given
 
 
@@ -64,7 +64,7 @@ def test_rounding_hook_rounds_what_it_is_told_and_nothing_else():
     is_bf16 = lambda a: np.array_equal(round_bf16(a), a)
     for name in ("Z", "H", "X_out"):
         assert is_bf16(ff[name]), name
-    for name in ("dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2"):
+    for name in ("dX_e", "dZ", "dX_in", "dL", "dX", "dWg", "dW1", "dW2", "db1", "db2"):
         assert is_bf16(fb[name]), name
     for name, a in (("X_e", ff["X_e"]), ("dG", fb["dG"]), ("dH", fb["dH"])):
         assert not is_bf16(a), name                          # left in fp64
