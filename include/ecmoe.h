@@ -224,6 +224,9 @@ ec_status ec_route_static(const ec_config* cfg, const void* X, const void* Wg, f
  * slots (i, j) holding t of G[i, j] * X_e[i, j, :], experts in ascending order, in
  * fp32, rounded once.  Rows of tokens that no expert chose are zero.
  *   W1, W2 [E, d, d'] (W2 is applied transposed);  X_out [n, d] out.
+ * b1 [E, d'] and b2 [E, d] (cfg->dtype, 16-byte aligned) are the bias terms the paper leaves out of Eq. 3 "for
+ * brevity": X_e[i] = GeLU(X_in[i] . W1[i] + b1[i]) . W2[i]^T + b2[i].  Either may be NULL (no such term: the equation
+ * as printed).
  * `saved` (ec_saved_bytes(cfg) bytes, 256-byte aligned) receives what the backward
  * pass needs (the intermediates live there).  Forward only (inference): pass saved = NULL
  * and saved_bytes = 0; the intermediates then live in `ws`, which must hold
@@ -231,20 +234,23 @@ ec_status ec_route_static(const ec_config* cfg, const void* X, const void* Wg, f
  * pass reads, is not written at all.  X_out is the same, bit for bit.
  */
 ec_status ec_moe_forward(const ec_config* cfg, const void* X, const void* Wg, const void* W1,
-                         const void* W2, void* X_out, void* saved, size_t saved_bytes, void* ws,
-                         size_t ws_bytes, void* cuda_stream);
+                         const void* W2, const void* b1, const void* b2, void* X_out, void* saved,
+                         size_t saved_bytes, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * Backward of Eq. 2-4 (the paper trains the gate, Section 3.4, and leaves the
  * derivative to automatic differentiation): gradients of <dX_out, X_out> with I held
  * constant, so the gate receives gradient through G only.
  *   dX_out [n, d] in, `saved` as filled by ec_moe_forward with the same cfg and inputs;
- *   dX [n, d], dWg [d, E], dW1, dW2 [E, d, d'] out, overwritten (not accumulated).
+ *   dX [n, d], dWg [d, E], dW1, dW2 [E, d, d'] out, overwritten (not accumulated);
+ *   db1 [E, d'], db2 [E, d] out, the gradients of the bias terms (sums of dZ and of dX_e over an expert's slots,
+ *   in slot order, fp32, rounded once); either may be NULL (not wanted).  The biases themselves are not needed here:
+ *   the saved Z already contains b1.
  */
 ec_status ec_moe_backward(const ec_config* cfg, const void* X, const void* Wg, const void* W1,
                           const void* W2, const void* dX_out, const void* saved,
-                          size_t saved_bytes, void* dX, void* dWg, void* dW1, void* dW2, void* ws,
-                          size_t ws_bytes, void* cuda_stream);
+                          size_t saved_bytes, void* dX, void* dWg, void* dW1, void* dW2, void* db1,
+                          void* db2, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * One expert-batched product of Eq. 3 or of its backward on its own (benchmarks time the kernels apart from the layer

@@ -74,9 +74,9 @@ def lib():
         L.ec_shuffle.restype = C.c_int; L.ec_shuffle.argtypes = [P, V, V, V, V]
         L.ec_unshuffle.restype = C.c_int; L.ec_unshuffle.argtypes = [P, V, V, V, V, V, V]
         L.ec_moe_forward.restype = C.c_int
-        L.ec_moe_forward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, C.c_size_t, V]
+        L.ec_moe_forward.argtypes = [P, V, V, V, V, V, V, V, V, C.c_size_t, V, C.c_size_t, V]
         L.ec_moe_backward.restype = C.c_int
-        L.ec_moe_backward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, V, V, V, V, C.c_size_t, V]
+        L.ec_moe_backward.argtypes = [P, V, V, V, V, V, V, C.c_size_t, V, V, V, V, V, V, V, C.c_size_t, V]
         L.ec_read_status.restype = C.c_int; L.ec_read_status.argtypes = [V, V]
         L.ec_status_string.restype = C.c_char_p; L.ec_status_string.argtypes = [C.c_int]
         L.ec_uses_tensor_cores.restype = C.c_int; L.ec_uses_tensor_cores.argtypes = [P]
@@ -258,33 +258,35 @@ def ec_route_static(cfg, X, Wg, out: Routing) -> Routing:
     return out
 
 
-def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None, forward_only=False):
-    """Eq. 2-4.  Returns (X_out, saved); with forward_only nothing is kept for a backward pass (saved is None)."""
+def ec_moe_forward(cfg, X, Wg, W1, W2, X_out=None, saved=None, ws=None, forward_only=False, b1=None, b2=None):
+    """Eq. 2-4.  Returns (X_out, saved); with forward_only nothing is kept for a backward pass (saved is None).
+    b1 [E, d'], b2 [E, d]: the bias terms Eq. 3 leaves out (None = none)."""
     dev = X.device
     X_out = torch.empty(total_tokens(cfg), cfg.d_model, dtype=_torch_dtype(cfg), device=dev) if X_out is None else X_out
     if forward_only:
         nb = int(lib().ec_forward_only_workspace_bytes(C.byref(cfg)))
         if ws is None or ws.numel() < nb:
             ws = torch.empty(nb, dtype=torch.uint8, device=dev)
-        _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),
+        _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(b1), _ptr(b2), _ptr(X_out),
                                     None, 0, _ptr(ws), ws.numel(), _stream()), "ec_moe_forward")
         return X_out, None
     saved = alloc_saved(cfg, dev) if saved is None else saved
     ws = alloc_workspace(cfg, dev) if ws is None else ws
-    _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(X_out),
+    _check(lib().ec_moe_forward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(b1), _ptr(b2), _ptr(X_out),
                                 _ptr(saved), saved.numel(), _ptr(ws), ws.numel(), _stream()), "ec_moe_forward")
     return X_out, saved
 
 
-def ec_moe_backward(cfg, X, Wg, W1, W2, dX_out, saved, grads=None, ws=None):
-    """Backward of Eq. 2-4.  Returns (dX, dWg, dW1, dW2)."""
+def ec_moe_backward(cfg, X, Wg, W1, W2, dX_out, saved, grads=None, ws=None, bias_grads=None):
+    """Backward of Eq. 2-4.  Returns (dX, dWg, dW1, dW2).  bias_grads = (db1 [E, d'], db2 [E, d]) are filled when given."""
     dev = X.device
     if grads is None:
         grads = (torch.empty_like(X), torch.empty_like(Wg), torch.empty_like(W1), torch.empty_like(W2))
     dX, dWg, dW1, dW2 = grads
     ws = alloc_workspace(cfg, dev) if ws is None else ws
+    db1, db2 = bias_grads if bias_grads is not None else (None, None)
     _check(lib().ec_moe_backward(C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(W1), _ptr(W2), _ptr(dX_out),
-                                 _ptr(saved), saved.numel(), _ptr(dX), _ptr(dWg), _ptr(dW1), _ptr(dW2),
+                                 _ptr(saved), saved.numel(), _ptr(dX), _ptr(dWg), _ptr(dW1), _ptr(dW2), _ptr(db1), _ptr(db2),
                                  _ptr(ws), ws.numel(), _stream()), "ec_moe_backward")
     return dX, dWg, dW1, dW2
 

@@ -146,6 +146,7 @@ struct BatchedGemm {
   void* C2; const void* Zin;
   int c_f32;                                         // C is fp32 regardless of the path's dtype
   const int32_t* batch_rows; int ragged;             // see TcGemmArgs: meaningful rows per batch along M (1) or K (2)
+  const void* bias;                                  // [batches, N] of the path's dtype, added to the accumulator (Eq. 3's omitted bias terms)
 };
 
 ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaStream_t st) {
@@ -156,7 +157,7 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
     t.lda = b.lda; t.ldb = b.ldb; t.batch_a = b.batch_a; t.batch_b = b.batch_b;
     t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c; t.c_f32 = b.c_f32;
     t.status = status_word;
-    t.batch_rows = b.batch_rows; t.ragged = b.ragged;
+    t.batch_rows = b.batch_rows; t.ragged = b.ragged; t.bias = b.bias;
     if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); return EC_OK; }
   }
   GemmArgs g; memset(&g, 0, sizeof(g));
@@ -167,6 +168,7 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
   g.sbk = b.b_mn ? b.ldb : 1; g.sbn = b.b_mn ? 1 : b.ldb;
   g.ldc = b.ldc; g.batch_a = b.batch_a; g.batch_b = b.batch_b; g.batch_c = b.batch_c;
   g.epi = b.epi; g.gelu = D.gelu; g.C2 = b.C2; g.Zin = b.Zin;
+  g.bias = b.bias; g.bias_dtype = D.dtype;
   EC_CUDA(launch_gemm_simt(g, st));
   return EC_OK;
 }
@@ -372,13 +374,14 @@ ec_status ec_route_static(const ec_config* c, const void* X, const void* Wg, flo
 }
 
 ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, const void* W1, const void* W2,
-                         void* X_out, void* saved, size_t saved_bytes, void* ws, size_t ws_bytes, void* stream) {
+                         const void* b1, const void* b2, void* X_out, void* saved, size_t saved_bytes, void* ws,
+                         size_t ws_bytes, void* stream) {
   Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
   if (!X || !Wg || !W1 || !W2 || !X_out || !ws) return EC_ERR_INVALID_ARG;
   const bool keep = saved != nullptr;                // else forward only: nothing is kept for a backward pass
   if (!keep && saved_bytes != 0) return EC_ERR_INVALID_ARG;
   if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(W1, 16) || misaligned(W2, 16) || misaligned(X_out, 16) ||
-      misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+      misaligned(b1, 16) || misaligned(b2, 16) || misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
   const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D, keep);
   if (keep ? (ws_bytes < W.total || saved_bytes < L.total) : ws_bytes < W.fwd_end + L.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
@@ -399,11 +402,11 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   prof_mark("gather", st);
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Z = X_in[i] . W1[i],  H = GeLU(Z)
-  BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr, 0, rag, 1};
+  BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr, 0, rag, 1, b1};
   if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
   prof_mark("gemm1_gelu", st);
   // X_e = H[i] . W2[i]^T, kept in fp32
-  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1, rag, 1};
+  BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1, rag, 1, b2};
   if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
   prof_mark("gemm2", st);
   EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
@@ -413,12 +416,12 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
 
 ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, const void* W1, const void* W2,
                           const void* dX_out, const void* saved, size_t saved_bytes, void* dX, void* dWg,
-                          void* dW1, void* dW2, void* ws, size_t ws_bytes, void* stream) {
+                          void* dW1, void* dW2, void* db1, void* db2, void* ws, size_t ws_bytes, void* stream) {
   Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
   if (!X || !Wg || !W1 || !W2 || !dX_out || !saved || !dX || !dWg || !dW1 || !dW2 || !ws) return EC_ERR_INVALID_ARG;
   if (misaligned(X, 16) || misaligned(Wg, 16) || misaligned(W1, 16) || misaligned(W2, 16) || misaligned(dX_out, 16) ||
       misaligned(dX, 16) || misaligned(dWg, 16) || misaligned(dW1, 16) || misaligned(dW2, 16) ||
-      misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+      misaligned(db1, 16) || misaligned(db2, 16) || misaligned(saved, kAlign) || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
   const WsLayout W = ws_layout(D); const SavedLayout L = saved_layout(D);
   if (ws_bytes < W.total || saved_bytes < L.total) return EC_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
@@ -438,19 +441,24 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
   prof_mark("bwd_combine", st);
   // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
-  BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z, 0, rag, 1};
+  BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z, 0, rag, 1, nullptr};
   if ((s = run_gemm(D, g3, status, st)) != EC_OK) return s;
   prof_mark("gemm_dZ", st);
+  if (db1 || db2) {                                  // gradients of the bias terms: sums over an expert's slots of dZ and of dX_e
+    if (db1) EC_CUDA(launch_column_sums(D.dtype, dZ, db1, D.E, D.k, D.dff, rag, st));
+    if (db2) EC_CUDA(launch_column_sums(D.dtype, dX_e, db2, D.E, D.k, D.d, rag, st));
+    prof_mark("bias_grads", st);
+  }
   // dW2[i] = dX_e[i]^T . H[i]
-  BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2};
+  BatchedGemm g4 = {dX_e, 1, D.d, kd, H, 1, D.dff, kf, dW2, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2, nullptr};
   if ((s = run_gemm(D, g4, status, st)) != EC_OK) return s;
   prof_mark("gemm_dW2", st);
   // dW1[i] = X_in[i]^T . dZ[i]
-  BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2};
+  BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2, nullptr};
   if ((s = run_gemm(D, g5, status, st)) != EC_OK) return s;
   prof_mark("gemm_dW1", st);
   // dX_in[i] = dZ[i] . W1[i]^T
-  BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 1};
+  BatchedGemm g6 = {dZ, 0, D.dff, kf, W1, 0, D.dff, df, dX_in, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 1, nullptr};
   if ((s = run_gemm(D, g6, status, st)) != EC_OK) return s;
   prof_mark("gemm_dXin", st);
   // softmax backward: dL [n, E]; bf16 when the two gate-gradient products below run on tensor cores
@@ -513,9 +521,9 @@ ec_status ec_expert_gemm(const ec_config* c, int kind, const void* A, const void
   EC_CUDA(cudaMemsetAsync(ws, 0, sizeof(StatusWord), st));
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   BatchedGemm g;
-  if (kind == EC_GEMM_XW1) g = {A, 0, D.d, kd, B, 1, D.dff, df, C, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
-  else if (kind == EC_GEMM_HW2T) g = {A, 0, D.dff, kf, B, 0, D.dff, df, C, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
-  else g = {A, 1, D.d, kd, B, 1, D.dff, kf, C, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0};
+  if (kind == EC_GEMM_XW1) g = {A, 0, D.d, kd, B, 1, D.dff, df, C, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0, nullptr};
+  else if (kind == EC_GEMM_HW2T) g = {A, 0, D.dff, kf, B, 0, D.dff, df, C, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0, nullptr};
+  else g = {A, 1, D.d, kd, B, 1, D.dff, kf, C, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, nullptr, 0, nullptr};
   prof_begin(st, 0);
   s = run_gemm(D, g, (int*)ws, st);
   prof_mark("expert_gemm", st);

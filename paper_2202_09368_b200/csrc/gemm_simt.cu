@@ -86,6 +86,7 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
       if (n >= g.N) continue;
       const int64_t o = (int64_t)m * g.ldc + n;
       float v = acc[i][j];
+      if (g.bias) v += g.bias_dtype == 0 ? ((const float*)g.bias)[(int64_t)b * g.N + n] : __bfloat162float(((const bf16*)g.bias)[(int64_t)b * g.N + n]);
       if (g.epi == EPI_GELU) {
         stv((TC*)g.C2 + (int64_t)b * g.batch_c, o, gelu_fwd(v, g.gelu));
       } else if (g.epi == EPI_GELU_GRAD) {

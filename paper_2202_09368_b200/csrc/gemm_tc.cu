@@ -90,6 +90,7 @@ struct TcParams {
   int skip_c;                                        // EPI_GELU: only H = GeLU(acc) is stored, the accumulator itself is not
   const int32_t* row_ptr; const int32_t* slots; const bf16* rows; int64_t ld_rows;   // EPI_ADD_SLOTS
   const int32_t* batch_rows; int ragged;             // meaningful rows per batch along M (1) or K (2), zeros beyond
+  const bf16* bias;                                  // EPI_GELU, EPI_STORE_F32: bias[b * N + n] joins every row of the accumulator
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -574,6 +575,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int c0 = half * kColsPerWarp; active && c0 < (half + 1) * kColsPerWarp; c0 += 32, ++nchunk) {
             if (n0 + c0 >= p.N) break;             // uniform across the warp
             uint32_t r[32]; tc_ld32(taddr + c0, r);
+            if (p.bias != nullptr) {               // the bias term of Eq. 3's second product: the same 32 values for every row
+              const bf16* bp = p.bias + (int64_t)b * p.N + n0 + c0;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                if (n0 + c0 + 8 * j < p.N) {
+                  const uint4 bv = __ldg(reinterpret_cast<const uint4*>(bp + 8 * j));
+                  const unsigned w[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) + __uint_as_float(w[e] << 16));
+                    r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) + __uint_as_float(w[e] & 0xFFFF0000u));
+                  }
+                }
+              }
+            }
             uint8_t* bufp = stg + (nchunk & 1) * 4096;
             if (lane == 0) bulk_wait_read<1>();
             __syncwarp();
@@ -592,6 +608,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t r[64];
             tc_ld32_issue(taddr + c0, r); tc_ld32_issue(taddr + c0 + 32, r + 32); tc_ld_wait();
             if constexpr (EPI == EPI_GELU) {
+              if (p.bias != nullptr) {             // Z = X_in . W1 + b1: the same 64 values for every row
+                const bf16* bp = p.bias + (int64_t)b * p.N + n0 + c0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  if (n0 + c0 + 8 * j < p.N) {
+                    const uint4 bv = __ldg(reinterpret_cast<const uint4*>(bp + 8 * j));
+                    const unsigned w[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      r[8 * j + 2 * e] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e]) + __uint_as_float(w[e] << 16));
+                      r[8 * j + 2 * e + 1] = __float_as_uint(__uint_as_float(r[8 * j + 2 * e + 1]) + __uint_as_float(w[e] & 0xFFFF0000u));
+                    }
+                  }
+                }
+              }
               // both buffers are written: Z into the first, H = GeLU(Z) into the second
               if (lane == 0) bulk_wait_read<0>();
               __syncwarp();
@@ -842,6 +873,7 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
                                  ((uintptr_t)g.rows & 15))) return false;
   if ((int64_t)g.lda * 2 >= ((int64_t)1 << 40) || (int64_t)g.ldb * 2 >= ((int64_t)1 << 40)) return false;
   if (g.batch_rows && (g.k_split || (g.ragged != 1 && g.ragged != 2))) return false;
+  if (g.bias && (((uintptr_t)g.bias & 15) || g.k_split || !(g.epi == EPI_GELU || (g.epi == EPI_STORE && g.c_f32)))) return false;
   return true;
 }
 
@@ -888,6 +920,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.n_fast = (int64_t)g.M * g.N > ((int64_t)g.M + g.N) * g.K ? 1 : 0;
   p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows;
   p.batch_rows = g.batch_rows; p.ragged = g.ragged;
+  p.bias = (const bf16*)g.bias;
   switch (g.epi) {
     case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
                                    : launch_bn<EPI_STORE>(bn, ctas, ta, tb, tc, tc2, p, st);

@@ -60,6 +60,10 @@ cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, 
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr,
                                const int32_t* slots, void* dL, int dl_bf16, int64_t n, int E, int64_t k,
                                cudaStream_t st);
+// out[b, c] = sum over the rows r < min(rows, batch_rows[b]) of A[b, r, c], in ascending r, fp32, cast to dtype
+// (gradients of the bias terms: column sums of dZ and dX_e per expert); batch_rows may be null
+cudaError_t launch_column_sums(int dtype, const void* A, void* out, int batches, int64_t rows, int cols,
+                               const int32_t* batch_rows, cudaStream_t st);
 // out[r,c] = sum_p part[p,r,c] in ascending p (fixed order), cast to dtype
 cudaError_t launch_reduce_partials(int dtype, const float* part, void* out, int P, int64_t elems,
                                    cudaStream_t st);
@@ -88,6 +92,7 @@ struct GemmArgs {
   void* C2;                            // EPI_GELU: receives GeLU(acc) (C receives acc, unless C is null)
   const void* Zin;                     // EPI_GELU_GRAD: C = acc * GeLU'(Zin), same layout and dtype as C
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;  // EPI_ADD_SLOTS
+  const void* bias; int bias_dtype;    // not null: bias[b * N + n] is added to the accumulator before the epilogue's function
 };
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 
@@ -118,6 +123,9 @@ struct TcGemmArgs {
   // first one, so rows 0 .. tile-1 of C are always written).  ragged = 2: it is K; k-blocks that start at or beyond
   // batch_rows[b] are skipped (at least one is run).
   const int32_t* batch_rows; int ragged;
+  // bias != null (EPI_GELU, or EPI_STORE with fp32 C): bf16 bias[b * N + n] is added to every row of the accumulator
+  // before the epilogue's function (the bias terms Eq. 3 leaves out); 16-byte aligned.
+  const void* bias;
 };
 constexpr int EPI_SOFTMAX = 4;
 bool tc_gemm_supported(const TcGemmArgs& g);

@@ -1159,6 +1159,40 @@ cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* r
 }
 
 // ------------------------------------------------------------------------------------------
+// Column sums per expert (gradients of the bias terms Eq. 3 leaves out): a thread owns a column and adds its rows in
+// order, so the result does not depend on scheduling; neighbouring threads read neighbouring columns.
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) column_sums_kernel(const T* __restrict__ A, T* __restrict__ out, int64_t rows, int cols,
+                                                          const int32_t* __restrict__ batch_rows) {
+  const int b = blockIdx.y, c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= cols) return;
+  int64_t lim = rows;
+  if (batch_rows != nullptr && batch_rows[b] < lim) lim = batch_rows[b];
+  const T* p = A + (int64_t)b * rows * cols + c;
+  float acc = 0.f;
+  int64_t r = 0;
+  for (; r + 8 <= lim; r += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = ld_f(p, (r + u) * cols);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += v[u];
+  }
+  for (; r < lim; ++r) acc += ld_f(p, r * cols);
+  if constexpr (sizeof(T) == 4) out[(int64_t)b * cols + c] = acc; else out[(int64_t)b * cols + c] = __float2bfloat16(acc);
+}
+
+cudaError_t launch_column_sums(int dtype, const void* A, void* out, int batches, int64_t rows, int cols,
+                               const int32_t* batch_rows, cudaStream_t st) {
+  const dim3 grid((cols + 255) / 256, batches);
+  count_launch();
+  if (dtype == 0) column_sums_kernel<float><<<grid, 256, 0, st>>>((const float*)A, (float*)out, rows, cols, batch_rows);
+  else column_sums_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)A, (bf16*)out, rows, cols, batch_rows);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
 // Fixed-order sum of split partial results.
 // ------------------------------------------------------------------------------------------
 template <typename T>

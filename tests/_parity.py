@@ -115,15 +115,19 @@ def check_routing(cfg, S_gpu, I_gpu, G_gpu, row_ptr, slots):
     return I_ref
 
 
-def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1, router="expert", **cap):
+def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S=True, groups=1, router="expert",
+                  biases=None, **cap):
     """Runs forward (+ backward) on the GPU and checks every tensor against the oracle.
-    n is the number of tokens per routing group; li holds groups * n rows."""
+    n is the number of tokens per routing group; li holds groups * n rows.  biases = (b1 [E, d'], b2 [E, d]) turns on
+    the bias terms Eq. 3 leaves out, and their gradients are then checked too."""
     tol = TOL[dtype]
     cfg = B.make_config(n, d, dff, E, c, dtype, gelu, groups=groups, router=router, **cap)
     dev = "cuda"
     X, Wg, W1, W2 = (t.to(dev) for t in (li.X, li.Wg, li.W1, li.W2))
     ws = B.alloc_workspace(cfg)
-    X_out, saved = B.ec_moe_forward(cfg, X, Wg, W1, W2, ws=ws)
+    b1, b2 = (t.to(dev) for t in biases) if biases is not None else (None, None)
+    b1n, b2n = (to_np(t) for t in biases) if biases is not None else (None, None)
+    X_out, saved = B.ec_moe_forward(cfg, X, Wg, W1, W2, ws=ws, b1=b1, b2=b2)
     assert B.ec_read_status(ws) == B.EC_OK
     v = B.saved_view(cfg, saved)
     Xn, Wgn, W1n, W2n = (to_np(t) for t in (li.X, li.Wg, li.W1, li.W2))
@@ -136,13 +140,15 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
     else:
         check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
     f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(), groups=groups,
-                  router=router)
+                  router=router, b1=b1n, b2=b2n)
     assert np.array_equal(v["X_in"].float().cpu().numpy(), f["X_in"].astype(np.float32))    # the shuffle of Eq. 3 is a copy
     filled = v["I"].cpu().numpy() >= 0             # all slots with expert choice; token choice leaves some empty, and
     got = {}                                       # what the library keeps for an empty slot is unspecified
     for name in ("Z", "H", "X_e"):
         got[name] = to_np(v[name])
         got[name][~filled] = 0.0
+        if biases is not None:
+            f[name] = np.where(filled[:, :, None], f[name], 0.0)       # with biases the oracle's empty slots are not zero either
         errs[name] = rel_err(got[name], f[name])
     got["X_out"] = to_np(X_out)
     errs["X_out"] = rel_err(got["X_out"], f["X_out"])
@@ -150,10 +156,14 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
     assert torch.all(X_out[torch.from_numpy(cnt == 0).to(dev)] == 0)
     if backward:
         dY = li.dX_out.to(dev)
-        dX, dWg, dW1, dW2 = B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, ws=ws)
+        bg = None
+        if biases is not None:
+            bg = (torch.empty(E, dff, dtype=dtype, device=dev), torch.empty(E, d, dtype=dtype, device=dev))
+        dX, dWg, dW1, dW2 = B.ec_moe_backward(cfg, X, Wg, W1, W2, dY, saved, ws=ws, bias_grads=bg)
         assert B.ec_read_status(ws) == B.EC_OK
         b = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), f, gelu)
-        for name, t in (("dX", dX), ("dWg", dWg), ("dW1", dW1), ("dW2", dW2)):
+        outs = [("dX", dX), ("dWg", dWg), ("dW1", dW1), ("dW2", dW2)] + ([("db1", bg[0]), ("db2", bg[1])] if bg else [])
+        for name, t in outs:
             got[name] = to_np(t)
             errs[name] = rel_err(got[name], b[name])
     bound = {k_: tol for k_ in errs}
@@ -161,7 +171,7 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
     if dtype == torch.bfloat16:
         rec = Bf16Recorder()
         ff = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(),
-                       store=rec, groups=groups, router=router)
+                       store=rec, groups=groups, router=router, b1=b1n, b2=b2n)
         refs = dict(f)
         if backward:
             fb = O.backward(Xn, Wgn, W1n, W2n, to_np(li.dX_out), ff, gelu, store=rec)
@@ -170,7 +180,10 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         detail, bad = {}, {k_: v_ for k_, v_ in bad.items() if k_ == "S"}
         for k_, t in got.items():
             stored = k_ in BF16_STORED
-            a = bf16_assess(t, refs[k_], rec.before(k_, refs[k_]) if stored else ff[k_], stored, k_)
+            pre = rec.before(k_, refs[k_]) if stored else ff[k_]
+            if k_ in ("Z", "H", "X_e"):
+                pre = np.where(filled[:, :, None], pre, 0.0)           # empty slots are outside the comparison (see above)
+            a = bf16_assess(t, refs[k_], pre, stored, k_)
             detail[k_] = a
             if not a["ok"]:
                 bad[k_] = a

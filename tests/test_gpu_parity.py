@@ -120,6 +120,28 @@ def test_expert_gemm_on_its_own(dtype, n, d, dff, E):
             assert rel_err(got, ref) <= tol, kind
 
 
+@pytest.mark.parametrize("dtype,n,d,dff,E,c,router,groups", [
+    (F32, 300, 36, 100, 3, 1.5, "expert", 1),
+    (F32, 256, 32, 64, 4, 1.9, "token", 1),
+    (BF16, 1024, 128, 384, 8, 2.0, "expert", 1),
+    (BF16, 2048, 256, 2304, 4, 2.0, "expert", 2),      # 256 x 512 tiles in the second product, whose epilogue adds b2
+    (BF16, 4096, 128, 384, 4, 2.6, "token", 1),        # empty slots: their Z is b1, not zero, and must not reach any gradient
+])
+def test_bias_terms_forward_backward(dtype, n, d, dff, E, c, router, groups):
+    """The bias terms Eq. 3 leaves out "for brevity": Z = X_in . W1 + b1, X_e = H . W2^T + b2, and db1, db2."""
+    li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=29, expert_skew=1.0 if router == "token" else 0.0)
+    b1 = IN.normal_tensor((E, dff), 0.5, 29, IN.TID_AUX, dtype)
+    b2 = IN.normal_tensor((E, d), 0.5, 30, IN.TID_AUX, dtype)
+    errs = run_and_check(n, d, dff, E, c, dtype, li, groups=groups, router=router, biases=(b1, b2))
+    assert "db1" in errs and "db2" in errs
+    # without biases the same call gives a different output (the terms are really there)
+    cfg = B.make_config(n, d, dff, E, c, dtype, groups=groups, router=router)
+    X, Wg, W1, W2 = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2))
+    Y0, _ = B.ec_moe_forward(cfg, X, Wg, W1, W2, forward_only=True)
+    Y1, _ = B.ec_moe_forward(cfg, X, Wg, W1, W2, forward_only=True, b1=b1.cuda(), b2=b2.cuda())
+    assert not torch.equal(Y0, Y1)
+
+
 def test_read_status_maps_the_status_word():
     """ec_read_status only reads the first word of the workspace: 0 is EC_OK, 5 a bounded wait that expired, anything
     else is reported as a CUDA error.  No kernel is involved."""
@@ -173,7 +195,7 @@ def test_forward_only_gives_the_same_output_without_a_saved_blob(dtype, n, d, df
     # a workspace that is too small for the intermediates is refused before anything is launched
     small = torch.empty(B.ec_workspace_bytes(cfg) // 2 if dff > d else 256, dtype=torch.uint8, device="cuda")
     code = B.lib().ec_moe_forward(__import__("ctypes").byref(cfg), X.data_ptr(), Wg.data_ptr(), W1.data_ptr(), W2.data_ptr(),
-                                  Y_inf.data_ptr(), None, 0, small.data_ptr(), 256, None)
+                                  None, None, Y_inf.data_ptr(), None, 0, small.data_ptr(), 256, None)
     assert code == B.EC_ERR_WORKSPACE
     torch.cuda.synchronize()
 

@@ -59,7 +59,7 @@ def test_null_pointers_are_rejected_without_a_gpu():
     L = B.lib()
     code = L.ec_route(ctypes.byref(cfg), None, None, None, None, None, None, None, None, 0, None)
     assert code == B.EC_ERR_INVALID_ARG
-    code = L.ec_moe_forward(ctypes.byref(cfg), None, None, None, None, None, None, 0, None, 0, None)
+    code = L.ec_moe_forward(ctypes.byref(cfg), None, None, None, None, None, None, None, None, 0, None, 0, None)
     assert code == B.EC_ERR_INVALID_ARG
 
 
