@@ -55,7 +55,9 @@ typedef enum {
   EC_ERR_UNSUPPORTED = 2, /* a documented restriction is violated                                */
   EC_ERR_WORKSPACE = 3,   /* ws_bytes or saved_bytes smaller than required                       */
   EC_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (launch, tensor-map encode)    */
-  EC_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (reported by ec_read_status)     */
+  EC_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (reported by ec_read_status)     */
+  EC_ERR_INDEX = 6        /* debug build only: an index read from I, row_ptr or slots was out of
+                             range; the access was skipped (reported by ec_read_status)          */
 } ec_status;
 
 typedef enum { EC_F32 = 0, EC_BF16 = 1 } ec_dtype;
@@ -266,10 +268,27 @@ ec_status ec_expert_gemm(const ec_config* cfg, int kind, const void* A, const vo
                          size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Checks an index structure as ec_route / ec_route_token_choice produce it (the paper has no counterpart; for callers
+ * that build or modify I, row_ptr, slots themselves before ec_shuffle / ec_unshuffle, and for debugging): every entry
+ * of I [E, k] is a token of the slot's own routing group (or -1 with the token-choice router), row_ptr [n+1] starts at
+ * 0, never decreases and ends at the number of filled slots, and every token's list in `slots` is ascending, in range
+ * and points at slots that hold that token.  Any contents are safe to pass: every access is range-checked.  Writes
+ * the number of violations found to *violations (host memory) and synchronises `cuda_stream`.
+ */
+ec_status ec_validate_routing(const ec_config* cfg, const int32_t* I, const int32_t* row_ptr,
+                              const int32_t* slots, int64_t* violations, void* ws, size_t ws_bytes,
+                              void* cuda_stream);
+
+/* 1 if this library was built with -DEC_DEBUG: every kernel then range-checks each index it reads from I, row_ptr
+ * or slots before using it, skips the access when it is out of range and records EC_ERR_INDEX in the status word
+ * (ec_read_status).  The normal build compiles these checks out. */
+int ec_debug_build(void);
+
+/*
  * Synchronises `cuda_stream` and reads the status word the kernels of the last call
  * on `ws` left there: EC_OK, or EC_ERR_TIMEOUT when a bounded wait inside a kernel
- * gave up (the outputs of that call are then undefined), or EC_ERR_CUDA when the
- * stream reports an error.
+ * gave up (the outputs of that call are then undefined), or EC_ERR_INDEX (debug build)
+ * when an index was out of range, or EC_ERR_CUDA when the stream reports an error.
  */
 ec_status ec_read_status(const void* ws, void* cuda_stream);
 

@@ -12,10 +12,12 @@ from dataclasses import dataclass
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libecmoe.so")
+# ECMOE_DEBUG=1 in the environment selects the build with index checks (python -m paper_2202_09368_b200.build --debug)
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                         "libecmoe_debug.so" if os.environ.get("ECMOE_DEBUG") == "1" else "libecmoe.so")
 _lib = None
 
-EC_OK, EC_ERR_INVALID_ARG, EC_ERR_UNSUPPORTED, EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT = range(6)
+EC_OK, EC_ERR_INVALID_ARG, EC_ERR_UNSUPPORTED, EC_ERR_WORKSPACE, EC_ERR_CUDA, EC_ERR_TIMEOUT, EC_ERR_INDEX = range(7)
 EC_F32, EC_BF16 = 0, 1
 EC_GELU_ERF, EC_GELU_TANH = 0, 1
 EC_ROUTER_EXPERT_CHOICE, EC_ROUTER_TOKEN_TOP2 = 0, 1
@@ -24,7 +26,7 @@ EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
            "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
-           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice", "ec_expert_gemm"]
+           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice", "ec_expert_gemm", "ec_validate_routing", "ec_debug_build"]
 EC_GEMM_XW1, EC_GEMM_HW2T, EC_GEMM_ATB = 0, 1, 2
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -67,6 +69,9 @@ def lib():
         L.ec_route_token_choice.argtypes = [P, V, V, V, V, V, V, V, V, V, V, C.c_size_t, V]
         L.ec_expert_gemm.restype = C.c_int
         L.ec_expert_gemm.argtypes = [P, C.c_int, V, V, V, V, C.c_size_t, V]
+        L.ec_validate_routing.restype = C.c_int
+        L.ec_validate_routing.argtypes = [P, V, V, V, C.POINTER(C.c_int64), V, C.c_size_t, V]
+        L.ec_debug_build.restype = C.c_int; L.ec_debug_build.argtypes = []
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
@@ -242,6 +247,19 @@ def ec_expert_gemm(cfg, kind, A, Bm, out=None, ws=None):
     _check(lib().ec_expert_gemm(C.byref(cfg), kind, _ptr(A), _ptr(Bm), _ptr(out), _ptr(ws), ws.numel(), _stream()),
            "ec_expert_gemm")
     return out
+
+
+def ec_validate_routing(cfg, I, row_ptr, slots, ws=None) -> int:
+    """Number of violations found in an index structure (0 = consistent); synchronises the current stream."""
+    ws = alloc_workspace(cfg, I.device) if ws is None else ws
+    bad = C.c_int64(-1)
+    _check(lib().ec_validate_routing(C.byref(cfg), _ptr(I), _ptr(row_ptr), _ptr(slots), C.byref(bad), _ptr(ws), ws.numel(),
+                                     _stream()), "ec_validate_routing")
+    return int(bad.value)
+
+
+def ec_debug_build() -> bool:
+    return bool(lib().ec_debug_build())
 
 
 def ec_route_static_bytes(cfg: ec_config) -> int:

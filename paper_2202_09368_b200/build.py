@@ -1,7 +1,8 @@
 """Builds libecmoe.so (the C-ABI library) from csrc/ with nvcc for sm_100a, in-tree.
 
-Usage: python -m paper_2202_09368_b200.build [--force] [--verbose]
-Objects go to paper_2202_09368_b200/_build/, the library next to this file.
+Usage: python -m paper_2202_09368_b200.build [--force] [--verbose] [--debug]
+Objects go to paper_2202_09368_b200/_build/, the library next to this file.  --debug builds libecmoe_debug.so as well:
+the same sources with -DEC_DEBUG, in which every index a kernel reads from I, row_ptr or slots is range-checked.
 """
 from __future__ import annotations
 
@@ -26,7 +27,14 @@ def _newer(src_list, target):
     return any(os.path.getmtime(s) > t for s in src_list)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    out = build_one(force, verbose, OUT, OBJ, [])
+    if debug:
+        build_one(force, verbose, OUT.replace("libecmoe.so", "libecmoe_debug.so"), os.path.join(OBJ, "debug"), ["-DEC_DEBUG"])
+    return out
+
+
+def build_one(force, verbose, OUT, OBJ, extra) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "ecmoe.h"))
@@ -36,7 +44,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, s.replace(".cu", ".o"))
         objs.append(obj)
         if force or _newer([src] + headers, obj):
-            cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+            cmd = [NVCC] + FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
             procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for s, p in procs:
@@ -53,4 +61,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build("--force" in sys.argv, "--verbose" in sys.argv))
+    print(build("--force" in sys.argv, "--verbose" in sys.argv, "--debug" in sys.argv))

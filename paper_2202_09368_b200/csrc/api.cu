@@ -191,7 +191,7 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
     EC_CUDA(launch_token_top2(S, D.n, D.E, choice, st));
     EC_CUDA(launch_token_admit(S, choice, D.ng, D.E, D.kg, D.groups, I, G, load, requested, st));
     prof_mark("token_choice", st);
-    EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
+    EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, (int*)(ws + W.status), st));
     prof_mark("inverse_index", st);
     return EC_OK;
   }
@@ -204,9 +204,9 @@ ec_status route_impl(const Dims& D, const void* X, const void* Wg, float* S, int
     keys = A;
   }
   EC_CUDA(launch_topk(keys, D.ng, D.E, D.kg, D.groups, I, G, ws + W.topk, st));
-  if (D.cap_b) EC_CUDA(launch_gather_gate(S, I, G, D.slots, D.k, D.E, st));      // the gate weights stay S at I
+  if (D.cap_b) EC_CUDA(launch_gather_gate(S, I, G, D.slots, D.k, D.E, D.n, (int*)(ws + W.status), st));      // the gate weights stay S at I
   prof_mark("topk", st);
-  EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, st));
+  EC_CUDA(launch_inverse_index(I, D.n, D.slots, row_ptr, slots, ws + W.inverse, (int*)(ws + W.status), st));
   prof_mark("inverse_index", st);
   return EC_OK;
 }
@@ -331,7 +331,7 @@ ec_status ec_shuffle(const ec_config* c, const void* X, const int32_t* I, void* 
   if (misaligned(X, 16) || misaligned(I, 16) || misaligned(X_in, 16)) return EC_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   prof_begin(st, 0);
-  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
+  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, D.n, nullptr, st));
   prof_mark("gather", st);
   return EC_OK;
 }
@@ -344,7 +344,7 @@ ec_status ec_unshuffle(const ec_config* c, const float* X_e, const float* G, con
       misaligned(X_out, 16)) return EC_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   prof_begin(st, 0);
-  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
+  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, D.slots, nullptr, st));
   prof_mark("combine", st);
   return EC_OK;
 }
@@ -398,7 +398,7 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   int32_t* requested = D.router ? (int32_t*)(sv + L.requested) : nullptr;
   const int32_t* rag = D.router && D.groups == 1 ? load : nullptr;
   if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st, load, requested)) != EC_OK) return s;
-  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, st));
+  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, D.n, status, st));
   prof_mark("gather", st);
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Z = X_in[i] . W1[i],  H = GeLU(Z)
@@ -409,7 +409,7 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   BatchedGemm g2 = {H, 0, D.dff, kf, W2, 0, D.dff, df, X_e, D.d, kd, (int)D.k, D.d, D.dff, D.E, EPI_STORE, nullptr, nullptr, 1, rag, 1, b2};
   if ((s = run_gemm(D, g2, status, st)) != EC_OK) return s;
   prof_mark("gemm2", st);
-  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, st));
+  EC_CUDA(launch_combine(D.dtype, X_e, G, row_ptr, slots, X_out, D.n, D.d, D.slots, status, st));
   prof_mark("combine", st);
   return EC_OK;
 }
@@ -438,7 +438,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
   // Eq. 4 backward: dX_e, dG
   prof_begin(st, 1);
-  EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, st));
+  EC_CUDA(launch_bwd_combine(D.dtype, dX_out, X_e, G, I, dX_e, dG, D.slots, D.d, D.n, status, st));
   prof_mark("bwd_combine", st);
   // dZ = (dX_e[i] . W2[i]) * GeLU'(Z)
   BatchedGemm g3 = {dX_e, 0, D.d, kd, W2, 1, D.dff, df, dZ, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU_GRAD, nullptr, Z, 0, rag, 1, nullptr};
@@ -472,9 +472,9 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   tx.A = dL; tx.a_mn_major = 0; tx.lda = D.E; tx.B = Wg; tx.b_mn_major = 0; tx.ldb = D.E;
   tx.M = (int)D.n; tx.N = D.d; tx.K = D.E; tx.batches = 1;
   tx.epi = EPI_ADD_SLOTS; tx.C = dX; tx.ldc = D.d; tx.status = status;
-  tx.row_ptr = row_ptr; tx.slots = slots; tx.rows = dX_in; tx.ld_rows = D.d;
+  tx.row_ptr = row_ptr; tx.slots = slots; tx.rows = dX_in; tx.ld_rows = D.d; tx.slots_total = D.slots;
   const bool tc_gate = D.dtype == EC_BF16 && tc_gemm_supported(tw) && tc_gemm_supported(tx);
-  EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, tc_gate ? 1 : 0, D.n, D.E, D.k, st));
+  EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, tc_gate ? 1 : 0, D.n, D.E, D.k, status, st));
   prof_mark("bwd_softmax", st);
   if (tc_gate) {
     EC_CUDA(launch_gemm_tc(tw, st));
@@ -504,6 +504,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
     g.M = (int)D.n; g.N = D.d; g.K = D.E; g.batches = 1;
     g.sam = D.E; g.sak = 1; g.sbk = 1; g.sbn = D.E; g.ldc = D.d;
     g.epi = EPI_ADD_SLOTS; g.row_ptr = row_ptr; g.slots = slots; g.rows = dX_in; g.ld_rows = D.d;
+    g.slots_total = D.slots; g.status = status;
     EC_CUDA(launch_gemm_simt(g, st));
     prof_mark("dX", st);
   }
@@ -530,12 +531,36 @@ ec_status ec_expert_gemm(const ec_config* c, int kind, const void* A, const void
   return s;
 }
 
+ec_status ec_validate_routing(const ec_config* c, const int32_t* I, const int32_t* row_ptr, const int32_t* slots,
+                              int64_t* violations, void* ws, size_t ws_bytes, void* stream) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!I || !row_ptr || !slots || !violations || !ws || misaligned(ws, kAlign)) return EC_ERR_INVALID_ARG;
+  if (ws_bytes < ws_layout(D).total) return EC_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  int* counters = (int*)ws + 8;                        // inside the status block, past the words the kernels use
+  EC_CUDA(launch_validate_routing(I, row_ptr, slots, D.n, D.ng, D.E, D.k, D.kg, D.groups, D.router == EC_ROUTER_TOKEN_TOP2 ? 1 : 0,
+                                  counters, st));
+  int h[2] = {0, 0};
+  EC_CUDA(cudaMemcpyAsync(h, counters, sizeof(h), cudaMemcpyDeviceToHost, st));
+  EC_CUDA(cudaStreamSynchronize(st));
+  *violations = h[0];
+  return EC_OK;
+}
+
+int ec_debug_build(void) {
+#ifdef EC_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 ec_status ec_read_status(const void* ws, void* stream) {
   if (!ws) return EC_ERR_INVALID_ARG;
   StatusWord h;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return EC_ERR_CUDA;
   if (cudaMemcpy(&h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return EC_ERR_CUDA;
-  return h.code == 0 ? EC_OK : (h.code == EC_ERR_TIMEOUT ? EC_ERR_TIMEOUT : EC_ERR_CUDA);
+  return h.code == 0 ? EC_OK : (h.code == EC_ERR_TIMEOUT ? EC_ERR_TIMEOUT : (h.code == EC_ERR_INDEX ? EC_ERR_INDEX : EC_ERR_CUDA));
 }
 
 const char* ec_status_string(ec_status s) {
@@ -546,6 +571,7 @@ const char* ec_status_string(ec_status s) {
     case EC_ERR_WORKSPACE: return "workspace or saved buffer too small";
     case EC_ERR_CUDA: return "CUDA call failed";
     case EC_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case EC_ERR_INDEX: return "an index read from I, row_ptr or slots was out of range";
   }
   return "unknown status";
 }

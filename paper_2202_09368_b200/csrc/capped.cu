@@ -322,9 +322,11 @@ capped_resident_smem_kernel(const float* __restrict__ S, float* __restrict__ A, 
 }
 
 __global__ void gather_gate_kernel(const float* __restrict__ S, const int32_t* __restrict__ I, float* __restrict__ G,
-                                   int64_t slots_total, int64_t k, int E) {
-  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < slots_total; s += (int64_t)gridDim.x * blockDim.x)
-    G[s] = S[(int64_t)I[s] * E + (int)(s / k)];
+                                   int64_t slots_total, int64_t k, int E, int64_t n, int* status) {
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < slots_total; s += (int64_t)gridDim.x * blockDim.x) {
+    const int t = I[s];
+    G[s] = idx_ok(t, 0, n, status) ? S[(int64_t)t * E + (int)(s / k)] : 0.f;
+  }
 }
 
 int blocks_per_group(int64_t ng, int groups, int sms) {
@@ -448,10 +450,10 @@ cudaError_t launch_capped_assignment(const float* S, int64_t ng, int E, int64_t 
 }
 
 cudaError_t launch_gather_gate(const float* S, const int32_t* I, float* G, int64_t slots_total, int64_t k, int E,
-                               cudaStream_t st) {
+                               int64_t n, int* status, cudaStream_t st) {
   count_launch();
   const int64_t blocks = (slots_total + 255) / 256;
-  gather_gate_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(S, I, G, slots_total, k, E);
+  gather_gate_kernel<<<(unsigned)(blocks > 1184 ? 1184 : blocks), 256, 0, st>>>(S, I, G, slots_total, k, E, n, status);
   return cudaGetLastError();
 }
 

@@ -93,7 +93,12 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
         v *= gelu_bwd(ldv((const TC*)g.Zin + (int64_t)b * g.batch_c, o), g.gelu);
       } else if (g.epi == EPI_ADD_SLOTS) {
         const TC* rows = (const TC*)g.rows;
-        for (int q = g.row_ptr[m]; q < g.row_ptr[m + 1]; ++q) v += ldv(rows, (int64_t)g.slots[q] * g.ld_rows + n);
+        int qa = g.row_ptr[m], qb = g.row_ptr[m + 1];
+        if (!idx_ok(qa, 0, g.slots_total + 1, n == 0 ? g.status : nullptr) || !idx_ok(qb, qa, g.slots_total + 1, n == 0 ? g.status : nullptr)) qa = qb = 0;
+        for (int q = qa; q < qb; ++q) {
+          const int sid = g.slots[q];
+          if (idx_ok(sid, 0, g.slots_total, n == 0 ? g.status : nullptr)) v += ldv(rows, (int64_t)sid * g.ld_rows + n);
+        }
       }
       if (g.C) stv(C, o, v);                    // EPI_GELU without C: only GeLU(acc) is wanted
     }

@@ -89,6 +89,7 @@ struct TcParams {
   int k_split;                                       // batches are cuts of one product along K
   int skip_c;                                        // EPI_GELU: only H = GeLU(acc) is stored, the accumulator itself is not
   const int32_t* row_ptr; const int32_t* slots; const bf16* rows; int64_t ld_rows;   // EPI_ADD_SLOTS
+  int64_t slots_total;                               // rows of `rows`: what the debug build checks the slot ids against
   const int32_t* batch_rows; int ragged;             // meaningful rows per batch along M (1) or K (2), zeros beyond
   const bf16* bias;                                  // EPI_GELU, EPI_STORE_F32: bias[b * N + n] joins every row of the accumulator
 };
@@ -676,9 +677,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               if constexpr (EPI == EPI_ADD_SLOTS) {
                 // this thread's row gains the rows of its slots (128 bytes of each), in slot order
                 if (row_ok) {
-                  const int qa = p.row_ptr[row], qb = p.row_ptr[row + 1];
+                  int qa = p.row_ptr[row], qb = p.row_ptr[row + 1];
+                  if (!idx_ok(qa, 0, p.slots_total + 1, p.status) || !idx_ok(qb, qa, p.slots_total + 1, p.status)) qa = qb = 0;
                   for (int qq = qa; qq < qb; ++qq) {
-                    const bf16* src = p.rows + (int64_t)p.slots[qq] * p.ld_rows + n0 + c0;
+                    const int sid = p.slots[qq];
+                    if (!idx_ok(sid, 0, p.slots_total, p.status)) continue;
+                    const bf16* src = p.rows + (int64_t)sid * p.ld_rows + n0 + c0;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                       if (n0 + c0 + 8 * j < p.N) {
@@ -918,7 +922,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   // than the operands (short K: the weight gradients) the tiles run along N instead, so that what is written at
   // one time is whole rows of C rather than 512-byte pieces 2*N bytes apart, and they share the A tile.
   p.n_fast = (int64_t)g.M * g.N > ((int64_t)g.M + g.N) * g.K ? 1 : 0;
-  p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows;
+  p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows; p.slots_total = g.slots_total;
   p.batch_rows = g.batch_rows; p.ragged = g.ragged;
   p.bias = (const bf16*)g.bias;
   switch (g.epi) {

@@ -16,8 +16,23 @@ constexpr int kRadixPasses = 3;    // the 30 significant bits of a score in (0, 
 constexpr int kCandCap = 512;      // threshold-bucket keys per expert the final sort may choose from
 constexpr int kSortTile = 4096;    // 64-bit keys sorted in shared memory by one CTA
 
-// Word 0 of the workspace: status written by kernels (0 = fine, 5 = a bounded wait expired).
-struct StatusWord { int code; int where; int pad[62]; };
+// Word 0 of the workspace: status written by kernels (0 = fine, 5 = a bounded wait expired, 6 = an index read from
+// I, row_ptr or slots was out of range); word 2 counts such indices.
+struct StatusWord { int code; int where; int bad_indices; int pad[61]; };
+
+// Debug build (-DEC_DEBUG): every index read from I, row_ptr or slots is checked against its range before it is used;
+// a bad one is recorded in the status word and the access it would have addressed is skipped.  In the normal build
+// the check is compiled out.  `status` may be null (the stand-alone shuffle and unshuffle have no workspace): the bad
+// access is then skipped without a record.
+#ifdef EC_DEBUG
+__device__ __forceinline__ bool idx_ok(int64_t i, int64_t lo, int64_t hi, int* status) {
+  if (i >= lo && i < hi) return true;
+  if (status != nullptr) { atomicExch(status, 6); atomicAdd(status + 2, 1); }
+  return false;
+}
+#else
+__device__ __forceinline__ bool idx_ok(int64_t, int64_t, int64_t, int*) { return true; }
+#endif
 
 // Per-expert state of the radix selection.
 // prefix: key bits decided so far (bits below `shift` are open); k_rem: keys still wanted from the
@@ -45,21 +60,30 @@ cudaError_t launch_token_top2(const float* S, int64_t rows, int E, int32_t* choi
 cudaError_t launch_token_admit(const float* S, const int32_t* choice, int64_t n, int E, int64_t k, int groups,
                                int32_t* I, float* G, int32_t* load, int32_t* requested, cudaStream_t st);
 size_t inverse_scratch_bytes(int64_t n);
+// (`status`: the workspace's status word, for the index checks of the debug build; may be null)
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t slots_total, int32_t* row_ptr,
-                                 int32_t* slots, void* scratch, cudaStream_t st);
+                                 int32_t* slots, void* scratch, int* status, cudaStream_t st);
 cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t slots_total,
-                          int d, cudaStream_t st);
+                          int d, int64_t n, int* status, cudaStream_t st);
 cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const int32_t* row_ptr,
-                           const int32_t* slots, void* X_out, int64_t n, int d, cudaStream_t st);
+                           const int32_t* slots, void* X_out, int64_t n, int d, int64_t slots_total, int* status,
+                           cudaStream_t st);
+// Counts what is wrong with an index structure (every access range-checked): I entries outside [0, n) (or [-1, n) when
+// empty slots are allowed) or outside their routing group, row_ptr not starting at 0 / decreasing / not ending at
+// the number of filled slots, slots entries out of range, not ascending within a token, or pointing at a slot that
+// holds another token.  The count is added to *violations (device).
+cudaError_t launch_validate_routing(const int32_t* I, const int32_t* row_ptr, const int32_t* slots, int64_t n, int64_t ng,
+                                    int E, int64_t k_total, int64_t kg, int groups, int allow_empty, int* violations,
+                                    cudaStream_t st);
 // dX_e[s,:] = G[s] * dX_out[I[s],:],  dG[s] = <dX_out[I[s],:], X_e[s,:]>
 cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, const float* G,
-                               const int32_t* I, void* dX_e, float* dG, int64_t slots_total, int d,
-                               cudaStream_t st);
+                               const int32_t* I, void* dX_e, float* dG, int64_t slots_total, int d, int64_t n,
+                               int* status, cudaStream_t st);
 // dL[t,i] = S[t,i] * (dS[t,i] - sum_i' dS[t,i'] S[t,i']),  dS scattered from dG through the inverse index;
 // dL is stored as bf16 when dl_bf16 (operand of the tensor-core dWg / dX products), else fp32
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr,
                                const int32_t* slots, void* dL, int dl_bf16, int64_t n, int E, int64_t k,
-                               cudaStream_t st);
+                               int* status, cudaStream_t st);
 // out[b, c] = sum over the rows r < min(rows, batch_rows[b]) of A[b, r, c], in ascending r, fp32, cast to dtype
 // (gradients of the bias terms: column sums of dZ and dX_e per expert); batch_rows may be null
 cudaError_t launch_column_sums(int dtype, const void* A, void* out, int batches, int64_t rows, int cols,
@@ -76,7 +100,7 @@ cudaError_t launch_capped_assignment(const float* S, int64_t ng, int E, int64_t 
                                      float lambda, float* A, void* scratch, cudaStream_t st);
 // G[i, j] = S[I[i, j], i] for I, G of shape [E, k]
 cudaError_t launch_gather_gate(const float* S, const int32_t* I, float* G, int64_t slots_total, int64_t k, int E,
-                               cudaStream_t st);
+                               int64_t n, int* status, cudaStream_t st);
 
 // ---- plain FMA GEMM (gemm_simt.cu) -------------------------------------------------------------
 enum Epilogue { EPI_STORE = 0, EPI_GELU = 1, EPI_GELU_GRAD = 2, EPI_ADD_SLOTS = 3 };
@@ -92,6 +116,7 @@ struct GemmArgs {
   void* C2;                            // EPI_GELU: receives GeLU(acc) (C receives acc, unless C is null)
   const void* Zin;                     // EPI_GELU_GRAD: C = acc * GeLU'(Zin), same layout and dtype as C
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;  // EPI_ADD_SLOTS
+  int64_t slots_total; int* status;    // EPI_ADD_SLOTS, debug build: range of the slot ids and where a bad one is recorded
   const void* bias; int bias_dtype;    // not null: bias[b * N + n] is added to the accumulator before the epilogue's function
 };
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
@@ -118,6 +143,7 @@ struct TcGemmArgs {
   // EPI_ADD_SLOTS (bf16 C, batches == 1): C[m, :] = acc[m, :] + sum over q in [row_ptr[m], row_ptr[m+1]) of
   // rows[slots[q], :] in ascending q, summed in fp32 and rounded once.
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;
+  int64_t slots_total;               // EPI_ADD_SLOTS: number of rows of `rows` (the debug build checks the slot ids against it)
   // batch_rows != null: batch b holds only batch_rows[b] meaningful rows along its ragged dimension and zeros after
   // them.  ragged = 1: that dimension is M; row tiles that start at or beyond batch_rows[b] are skipped (never the
   // first one, so rows 0 .. tile-1 of C are always written).  ragged = 2: it is K; k-blocks that start at or beyond

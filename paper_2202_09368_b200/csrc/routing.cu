@@ -797,10 +797,10 @@ size_t inverse_scratch_bytes(int64_t n) {
   return inv_cnt_bytes(n) + ((((size_t)(n + kScanTile - 1) / kScanTile) * 4 + 255) & ~(size_t)255);
 }
 
-__global__ void inv_count_kernel(const int32_t* __restrict__ I, int64_t total, int32_t* cnt) {
+__global__ void inv_count_kernel(const int32_t* __restrict__ I, int64_t total, int32_t* cnt, int64_t n, int* status) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
     const int t = I[s];
-    if (t >= 0) atomicAdd(&cnt[t], 1);                 // -1: an empty slot (token-choice routing only)
+    if (t >= 0 && idx_ok(t, 0, n, status)) atomicAdd(&cnt[t], 1);      // -1: an empty slot (token-choice routing only)
   }
 }
 
@@ -855,10 +855,10 @@ __global__ void __launch_bounds__(kScanThreads) inv_scan_add_kernel(const int32_
 
 // Hands each slot a place in its token's list, counting the token's counter back down to zero.
 __global__ void inv_fill_kernel(const int32_t* __restrict__ I, int64_t total, const int32_t* __restrict__ row_ptr,
-                                int32_t* cnt, int32_t* slots) {
+                                int32_t* cnt, int32_t* slots, int64_t n) {
   for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) {
     const int t = I[s];
-    if (t >= 0) slots[row_ptr[t] + atomicSub(&cnt[t], 1) - 1] = (int32_t)s;
+    if (t >= 0 && idx_ok(t, 0, n, nullptr)) slots[row_ptr[t] + atomicSub(&cnt[t], 1) - 1] = (int32_t)s;   // counted once, in inv_count
   }
 }
 
@@ -878,13 +878,13 @@ __global__ void inv_sort_kernel(const int32_t* __restrict__ row_ptr, int64_t n, 
 // matter because every token's list is sorted at the end.
 constexpr int kInvSmallN = 4096, kInvSmallSlots = 1 << 14;
 __global__ void __launch_bounds__(1024)
-inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots) {
+inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots, int* status) {
   extern __shared__ int s_cnt[];                       // [n] counts, then cursors
   __shared__ int s_warp[33];
   const int tid = threadIdx.x;
   for (int t = tid; t < n; t += 1024) s_cnt[t] = 0;
   __syncthreads();
-  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0) atomicAdd(&s_cnt[t], 1); }
+  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0 && idx_ok(t, 0, n, status)) atomicAdd(&s_cnt[t], 1); }
   __syncthreads();
   // exclusive scan over the tokens, 1024 * per at a time
   const int per = (n + 1023) / 1024, a = min(n, tid * per), b = min(n, a + per);
@@ -895,7 +895,7 @@ inv_small_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_p
   for (int t = a; t < b; ++t) { const int c = s_cnt[t]; row_ptr[t] = run; s_cnt[t] = run; run += c; }   // s_cnt becomes the cursor
   if (tid == 0) row_ptr[n] = total_sum;
   __syncthreads();
-  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0) slots[atomicAdd(&s_cnt[t], 1)] = s; }
+  for (int s = tid; s < total; s += 1024) { const int t = I[s]; if (t >= 0 && idx_ok(t, 0, n, nullptr)) slots[atomicAdd(&s_cnt[t], 1)] = s; }
   __syncthreads();
   __threadfence_block();
   for (int t = tid; t < n; t += 1024) {                // after the fill s_cnt[t] is the end of token t's list
@@ -916,14 +916,14 @@ __device__ __forceinline__ void inv_cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __global__ void __launch_bounds__(1024)
-inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots, int32_t* cnt) {
+inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row_ptr, int32_t* slots, int32_t* cnt, int* status) {
   __shared__ int s_warp[33];
   __shared__ int s_tile;                               // sum of this CTA's part of the counts
   const int tid = threadIdx.x, rank = blockIdx.x, nc = gridDim.x;      // the grid is the one cluster
   const int gtid = rank * 1024 + tid, gsize = nc * 1024;
   for (int t = gtid; t < n; t += gsize) cnt[t] = 0;
   inv_cluster_sync();
-  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0) atomicAdd(&cnt[t], 1); }
+  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0 && idx_ok(t, 0, n, status)) atomicAdd(&cnt[t], 1); }
   inv_cluster_sync();
   // exclusive scan: CTA `rank` takes tokens [lo, hi), a thread `per` consecutive ones of them
   const int per_cta = (n + nc - 1) / nc, lo = min(n, rank * per_cta), hi = min(n, lo + per_cta);
@@ -945,7 +945,7 @@ inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row
   for (int t = a; t < b; ++t) { const int c = cnt[t]; row_ptr[t] = run; cnt[t] = run; run += c; }      // cnt becomes the cursor
   if (rank == nc - 1 && tid == 0) row_ptr[n] = before + tile;
   inv_cluster_sync();
-  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0) slots[atomicAdd(&cnt[t], 1)] = s; }
+  for (int s = gtid; s < total; s += gsize) { const int t = I[s]; if (t >= 0 && idx_ok(t, 0, n, nullptr)) slots[atomicAdd(&cnt[t], 1)] = s; }
   inv_cluster_sync();
   for (int t = gtid; t < n; t += gsize) {
     const int p0 = row_ptr[t], p1 = row_ptr[t + 1];
@@ -958,7 +958,7 @@ inv_cluster_kernel(const int32_t* __restrict__ I, int n, int total, int32_t* row
 }
 
 cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int32_t* row_ptr, int32_t* slots,
-                                 void* scratch, cudaStream_t st) {
+                                 void* scratch, int* status, cudaStream_t st) {
   if (n > kInvSmallN && n <= kInvClusterN && total <= kInvClusterSlots) {
     cudaLaunchConfig_t cfg; memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(kInvClusterCtas); cfg.blockDim = dim3(1024); cfg.stream = st;
@@ -967,14 +967,14 @@ cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int
     attr[0].val.clusterDim.x = kInvClusterCtas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     count_launch();
-    return cudaLaunchKernelEx(&cfg, inv_cluster_kernel, I, (int)n, (int)total, row_ptr, slots, (int32_t*)scratch);
+    return cudaLaunchKernelEx(&cfg, inv_cluster_kernel, I, (int)n, (int)total, row_ptr, slots, (int32_t*)scratch, status);
   }
   if (n <= kInvSmallN && total <= kInvSmallSlots) {
     const int smem = (int)n * 4;
     cudaError_t e0 = cudaFuncSetAttribute(inv_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e0 != cudaSuccess) return e0;
     count_launch();
-    inv_small_kernel<<<1, 1024, smem, st>>>(I, (int)n, (int)total, row_ptr, slots);
+    inv_small_kernel<<<1, 1024, smem, st>>>(I, (int)n, (int)total, row_ptr, slots, status);
     return cudaGetLastError();
   }
   int32_t* cnt = (int32_t*)scratch;
@@ -983,15 +983,74 @@ cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int
   cudaError_t e;
   if ((e = cudaMemsetAsync(cnt, 0, (size_t)(n + 1) * 4, st)) != cudaSuccess) return e;
   count_launch();
-  inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cnt);
+  inv_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, cnt, n, status);
   count_launch();
   inv_scan_tile_kernel<<<tiles, kScanThreads, 0, st>>>(cnt, n, row_ptr, tile_sum);
   count_launch();
   inv_scan_add_kernel<<<tiles, kScanThreads, 0, st>>>(tile_sum, n, row_ptr);
   count_launch();
-  inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cnt, slots);
+  inv_fill_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, total, row_ptr, cnt, slots, n);
   count_launch();
   inv_sort_kernel<<<grid_for(n, 256), 256, 0, st>>>(row_ptr, n, slots);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Validation of an index structure (on request, and what the debug build's checks are modelled on): every access
+// below is range-checked, so any contents are safe to hand in.  Violations are counted.
+// ------------------------------------------------------------------------------------------
+__global__ void validate_routing_kernel(const int32_t* __restrict__ I, const int32_t* __restrict__ row_ptr,
+                                        const int32_t* __restrict__ slots, int64_t n, int64_t ng, int E, int64_t k_total,
+                                        int64_t kg, int groups, int allow_empty, int* violations) {
+  const int64_t total = (int64_t)E * k_total;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x, g0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  int bad = 0;
+  // slots: a token of the slot's own routing group, or -1 where empty slots exist
+  for (int64_t s = g0; s < total; s += stride) {
+    const int t = I[s];
+    const int64_t grp = (s % k_total) / kg;
+    if (t == -1) { if (!allow_empty) ++bad; }
+    else if (t < 0 || t >= n || t / ng != grp) ++bad;
+  }
+  // the token -> slot lists
+  for (int64_t t = g0; t < n; t += stride) {
+    const int64_t a = row_ptr[t], b = row_ptr[t + 1];
+    if (t == 0 && a != 0) ++bad;
+    if (a < 0 || b < a || b > total) { ++bad; continue; }
+    int prev = -1;
+    for (int64_t q = a; q < b; ++q) {
+      const int s = slots[q];
+      if (s < 0 || s >= total) { ++bad; continue; }
+      if (s <= prev) ++bad;                             // ascending slot ids, hence ascending expert
+      if (I[s] != t) ++bad;
+      prev = s;
+    }
+  }
+  if (bad) atomicAdd(violations, bad);
+}
+
+// every filled slot is listed exactly once: row_ptr[n] equals the number of filled slots
+__global__ void validate_count_kernel(const int32_t* __restrict__ I, const int32_t* __restrict__ row_ptr, int64_t n, int64_t total,
+                                      int* filled) {
+  int c = 0;
+  for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (int64_t)gridDim.x * blockDim.x) c += I[s] >= 0;
+  if (c) atomicAdd(filled, c);
+}
+__global__ void validate_total_kernel(const int32_t* __restrict__ row_ptr, int64_t n, const int* filled, int* violations) {
+  if (row_ptr[n] != *filled) atomicAdd(violations, 1);
+}
+
+cudaError_t launch_validate_routing(const int32_t* I, const int32_t* row_ptr, const int32_t* slots, int64_t n, int64_t ng,
+                                    int E, int64_t k_total, int64_t kg, int groups, int allow_empty, int* violations,
+                                    cudaStream_t st) {
+  const int64_t total = (int64_t)E * k_total;
+  cudaError_t e = cudaMemsetAsync(violations, 0, 2 * sizeof(int), st);       // [0] violations, [1] filled slots
+  if (e != cudaSuccess) return e;
+  count_launch(3);
+  validate_routing_kernel<<<grid_for(total > n ? total : n, 256), 256, 0, st>>>(I, row_ptr, slots, n, ng, E, k_total, kg, groups,
+                                                                                 allow_empty, violations);
+  validate_count_kernel<<<grid_for(total, 256), 256, 0, st>>>(I, row_ptr, n, total, violations + 1);
+  validate_total_kernel<<<1, 1, 0, st>>>(row_ptr, n, violations + 1, violations);
   return cudaGetLastError();
 }
 
@@ -999,19 +1058,21 @@ cudaError_t launch_inverse_index(const int32_t* I, int64_t n, int64_t total, int
 // Shuffle, Eq. 3: X_in = P . X as an indexed row copy in 16-byte vectors.
 // ------------------------------------------------------------------------------------------
 __global__ void gather_kernel(const uint4* __restrict__ X, const int32_t* __restrict__ I, uint4* __restrict__ X_in,
-                              int64_t total_vec, int vec_per_row) {
+                              int64_t total_vec, int vec_per_row, int64_t n, int* status) {
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_vec; g += (int64_t)gridDim.x * blockDim.x) {
     const int64_t s = g / vec_per_row; const int v = (int)(g % vec_per_row);
-    const int t = I[s];                                // -1: an empty slot (token-choice routing only) holds a zero row
+    int t = I[s];                                      // -1: an empty slot (token-choice routing only) holds a zero row
+    if (t >= 0 && !idx_ok(t, 0, n, v == 0 ? status : nullptr)) t = -1;
     X_in[g] = t >= 0 ? X[(int64_t)t * vec_per_row + v] : make_uint4(0, 0, 0, 0);
   }
 }
 
-cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t total, int d, cudaStream_t st) {
+cudaError_t launch_gather(int dtype, const void* X, const int32_t* I, void* X_in, int64_t total, int d, int64_t n, int* status,
+                          cudaStream_t st) {
   const int vpr = d * (dtype == 0 ? 4 : 2) / 16;
   const int64_t tv = total * vpr;
   count_launch();
-  gather_kernel<<<grid_for(tv, 256, 148 * 32), 256, 0, st>>>((const uint4*)X, I, (uint4*)X_in, tv, vpr);
+  gather_kernel<<<grid_for(tv, 256, 148 * 32), 256, 0, st>>>((const uint4*)X, I, (uint4*)X_in, tv, vpr, n, status);
   return cudaGetLastError();
 }
 
@@ -1039,17 +1100,21 @@ __device__ __forceinline__ void store4(bf16* p, const float* f) {
 template <typename T>
 __global__ void combine_kernel(const float* __restrict__ X_e, const float* __restrict__ G,
                                const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
-                               T* __restrict__ X_out, int64_t total_quads, int quads_per_row) {
+                               T* __restrict__ X_out, int64_t total_quads, int quads_per_row, int64_t slots_total, int* status) {
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total_quads; g += (int64_t)gridDim.x * blockDim.x) {
     const int64_t t = g / quads_per_row; const int v = (int)(g % quads_per_row);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int a = row_ptr[t], b = row_ptr[t + 1];
+    int a = row_ptr[t], b = row_ptr[t + 1];
+    if (!idx_ok(a, 0, slots_total + 1, v == 0 ? status : nullptr) || !idx_ok(b, a, slots_total + 1, v == 0 ? status : nullptr)) a = b = 0;
     // four slots at a time: their ids, then their weights and row pieces, are fetched together, and
     // added in slot order
     for (int q0 = a; q0 < b; q0 += 4) {
       int s[4]; float w[4]; float4 x[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) s[u] = q0 + u < b ? slots[q0 + u] : -1;
+      for (int u = 0; u < 4; ++u) {
+        s[u] = q0 + u < b ? slots[q0 + u] : -1;
+        if (s[u] >= 0 && !idx_ok(s[u], 0, slots_total, v == 0 ? status : nullptr)) s[u] = -1;
+      }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         w[u] = s[u] >= 0 ? G[s[u]] : 0.f;
@@ -1068,12 +1133,12 @@ __global__ void combine_kernel(const float* __restrict__ X_e, const float* __res
 }
 
 cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const int32_t* row_ptr, const int32_t* slots,
-                           void* X_out, int64_t n, int d, cudaStream_t st) {
+                           void* X_out, int64_t n, int d, int64_t slots_total, int* status, cudaStream_t st) {
   const int qpr = d / 4;
   const int64_t tq = n * qpr;
   const unsigned grid = grid_for(tq, 256, 148 * 32);
-  if (dtype == 0) { count_launch(); combine_kernel<float><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (float*)X_out, tq, qpr); }
-  else { count_launch(); combine_kernel<bf16><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (bf16*)X_out, tq, qpr); }
+  if (dtype == 0) { count_launch(); combine_kernel<float><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (float*)X_out, tq, qpr, slots_total, status); }
+  else { count_launch(); combine_kernel<bf16><<<grid, 256, 0, st>>>(X_e, G, row_ptr, slots, (bf16*)X_out, tq, qpr, slots_total, status); }
   return cudaGetLastError();
 }
 
@@ -1084,11 +1149,13 @@ cudaError_t launch_combine(int dtype, const float* X_e, const float* G, const in
 template <typename T>
 __global__ void bwd_combine_kernel(const T* __restrict__ dX_out, const float* __restrict__ X_e,
                                    const float* __restrict__ G, const int32_t* __restrict__ I,
-                                   T* __restrict__ dX_e, float* __restrict__ dG, int64_t total, int quads_per_row) {
+                                   T* __restrict__ dX_e, float* __restrict__ dG, int64_t total, int quads_per_row, int64_t n,
+                                   int* status) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   for (int64_t s = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; s < total; s += warps) {
-    const int64_t t = I[s];
+    int64_t t = I[s];
+    if (t >= 0 && !idx_ok(t, 0, n, lane == 0 ? status : nullptr)) t = -1;
     if (t < 0) {                                       // an empty slot (token-choice routing only): zero row, no gradient
       const float z[4] = {0.f, 0.f, 0.f, 0.f};
       for (int v = lane; v < quads_per_row; v += 32) store4(dX_e + (s * quads_per_row + v) * 4, z);
@@ -1111,11 +1178,11 @@ __global__ void bwd_combine_kernel(const T* __restrict__ dX_out, const float* __
 }
 
 cudaError_t launch_bwd_combine(int dtype, const void* dX_out, const float* X_e, const float* G, const int32_t* I,
-                               void* dX_e, float* dG, int64_t total, int d, cudaStream_t st) {
+                               void* dX_e, float* dG, int64_t total, int d, int64_t n, int* status, cudaStream_t st) {
   const int qpr = d / 4;
   const unsigned grid = grid_for(total * 32, 256, 148 * 16);
-  if (dtype == 0) { count_launch(); bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)dX_out, X_e, G, I, (float*)dX_e, dG, total, qpr); }
-  else { count_launch(); bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)dX_out, X_e, G, I, (bf16*)dX_e, dG, total, qpr); }
+  if (dtype == 0) { count_launch(); bwd_combine_kernel<float><<<grid, 256, 0, st>>>((const float*)dX_out, X_e, G, I, (float*)dX_e, dG, total, qpr, n, status); }
+  else { count_launch(); bwd_combine_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)dX_out, X_e, G, I, (bf16*)dX_e, dG, total, qpr, n, status); }
   return cudaGetLastError();
 }
 
@@ -1129,14 +1196,17 @@ __device__ __forceinline__ void st_dl(bf16* p, int64_t i, float v) { p[i] = __fl
 template <typename TL>
 __global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __restrict__ dG,
                                    const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ slots,
-                                   TL* __restrict__ dL, int64_t n, int E, int64_t k) {
+                                   TL* __restrict__ dL, int64_t n, int E, int64_t k, int* status) {
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int64_t slots_total = (int64_t)E * k;
   for (int64_t t = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < n; t += warps) {
-    const int a = row_ptr[t], b = row_ptr[t + 1];
+    int a = row_ptr[t], b = row_ptr[t + 1];
+    if (!idx_ok(a, 0, slots_total + 1, lane == 0 ? status : nullptr) || !idx_ok(b, a, slots_total + 1, lane == 0 ? status : nullptr)) a = b = 0;
     float dot = 0.f;
     for (int q = a + lane; q < b; q += 32) {
       const int s = slots[q];
+      if (!idx_ok(s, 0, slots_total, status)) continue;
       dot = fmaf(dG[s], S[t * E + s / k], dot);
     }
     for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
@@ -1144,17 +1214,18 @@ __global__ void bwd_softmax_kernel(const float* __restrict__ S, const float* __r
     __syncwarp();
     for (int q = a + lane; q < b; q += 32) {           // the slots of one token belong to distinct experts
       const int s = slots[q]; const int64_t i = s / k;
+      if (!idx_ok(s, 0, slots_total, nullptr)) continue;
       st_dl(dL, t * E + i, S[t * E + i] * (dG[s] - dot));
     }
   }
 }
 
 cudaError_t launch_bwd_softmax(const float* S, const float* dG, const int32_t* row_ptr, const int32_t* slots,
-                               void* dL, int dl_bf16, int64_t n, int E, int64_t k, cudaStream_t st) {
+                               void* dL, int dl_bf16, int64_t n, int E, int64_t k, int* status, cudaStream_t st) {
   count_launch();
   const unsigned grid = grid_for(n * 32, 256, 148 * 16);
-  if (dl_bf16) bwd_softmax_kernel<bf16><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (bf16*)dL, n, E, k);
-  else bwd_softmax_kernel<float><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (float*)dL, n, E, k);
+  if (dl_bf16) bwd_softmax_kernel<bf16><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (bf16*)dL, n, E, k, status);
+  else bwd_softmax_kernel<float><<<grid, 256, 0, st>>>(S, dG, row_ptr, slots, (float*)dL, n, E, k, status);
   return cudaGetLastError();
 }
 
