@@ -133,10 +133,12 @@ def gemm_traffic(workload, E):
     digest = None
     for line in open(GEMM_PROFILE):
         cells = [c.strip() for c in line.split("|")]
-        if len(cells) > 3 and cells[1] == "dram__bytes_read.sum":
-            rd = [float(c) for c in cells[3:] if c]
-        if len(cells) > 3 and cells[1] == "dram__bytes_write.sum":
-            wr = [float(c) for c in cells[3:] if c]
+        if len(cells) > 3 and cells[1] in ("dram__bytes_read.sum", "dram__bytes_write.sum") and cells[2] == "Mbyte":
+            vals = [float(c) for c in cells[3:] if c]
+            if cells[1].endswith("read.sum"):
+                rd = vals
+            else:
+                wr = vals
         if line.startswith("kernel source digest:"):
             digest = line.split(":", 1)[1].strip().strip("`")
     if not rd or not wr or len(rd) != len(wr) or digest != source_digest():
@@ -479,6 +481,23 @@ def run_routing(args):
                     if it >= 3:
                         acc.setdefault(k_, []).append(v_)
         assert B.ec_read_status(ws) == B.EC_OK
+        # no case is printed whose output has not passed the checks that hold at any size (the parity tests compare
+        # these sizes with the oracle element by element; here: properties, on the device, with torch)
+        k = B.ec_capacity(cfg)
+        assert B.ec_validate_routing(cfg, r.I, r.row_ptr, r.slots, ws) == 0, "inconsistent index structure"
+        assert int(r.row_ptr[-1]) == E * k
+        cols = torch.arange(E, device=dev).unsqueeze(1).expand(E, k)
+        if not args.cap_b:
+            assert torch.equal(r.G, r.S[r.I.long(), cols]), "G is not S at the selected pairs"
+            chosen = torch.zeros(n, E, dtype=torch.bool, device=dev)
+            chosen[r.I.long(), cols] = True
+            assert int(chosen.sum()) == E * k, "an expert holds a token twice"
+            lowest_in = torch.where(chosen, r.S, torch.full_like(r.S, 2.0)).amin(dim=0)
+            highest_out = torch.where(chosen, torch.full_like(r.S, -1.0), r.S).amax(dim=0)
+            assert bool((lowest_in >= highest_out).all()), "a token outside an expert's top k scores higher than one inside"
+            assert bool((r.G[:, :-1] >= r.G[:, 1:]).all()), "an expert's slots are not in descending score order"
+            del chosen, lowest_in, highest_out
+        assert torch.equal(X_in, X[r.I.long()]), "the shuffle is not a copy of the selected rows"
         by = routing_bytes(n, d, E, c, cap_iters=args.cap_iters if args.cap_b else 0)
         st = {}
         for k_, v_ in acc.items():
@@ -498,7 +517,9 @@ def run_routing(args):
     B.ec_profile_enable(False)
     print(json.dumps({"metric": "ec_routing_chain", "unit": "GB/s (algorithmic bytes / device time per stage)",
                       "config": {"workload": "routing-only stress: d=1024 bf16 c=2, identity experts",
-                                 "l2": "512 MiB flush before every timed call"},
+                                 "l2": "512 MiB flush before every timed call",
+                                 "checked": "every case: status word, ec_validate_routing, G = S at I, k distinct tokens per expert, "
+                                            "threshold and order of every expert's scores, shuffle = row copy"},
                       "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "cases": cases}))
 
 

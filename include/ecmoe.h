@@ -284,6 +284,19 @@ ec_status ec_validate_routing(const ec_config* cfg, const int32_t* I, const int3
  * (ec_read_status).  The normal build compiles these checks out. */
 int ec_debug_build(void);
 
+/* Views into the workspace as ec_moe_backward leaves it (device pointers; valid until the next call that uses the
+ * workspace), for inspection and tests: the intermediates of the chain rule through Eq. 4, 3 and 2.  Rows of dZ and
+ * dX_in that belong to empty slots (token-choice router) are unspecified. */
+typedef struct {
+  void* dX_e;         /* [E, k, d]  G[i,j] * dX_out[I[i,j], :], cfg->dtype                       */
+  float* dG;          /* [E, k]     <dX_out[I[i,j], :], X_e[i,j,:]>                              */
+  void* dZ;           /* [E, k, d'] (dX_e[i] . W2[i]) * GeLU'(Z), cfg->dtype                     */
+  void* dX_in;        /* [E, k, d]  dZ[i] . W1[i]^T, cfg->dtype                                  */
+  void* dL;           /* [n, E]     gradient of the gate logits; bf16 if dL_is_bf16, else fp32   */
+  int32_t dL_is_bf16; /* 1 when the two gate-gradient products run on the tensor cores           */
+} ec_backward_ptrs;
+ec_status ec_backward_view(const ec_config* cfg, void* ws, ec_backward_ptrs* out);
+
 /*
  * Synchronises `cuda_stream` and reads the status word the kernels of the last call
  * on `ws` left there: EC_OK, or EC_ERR_TIMEOUT when a bounded wait inside a kernel

@@ -26,7 +26,7 @@ EXPORTS = ["ec_capacity", "ec_workspace_bytes", "ec_saved_bytes", "ec_saved_view
            "ec_moe_forward", "ec_moe_backward", "ec_read_status", "ec_status_string",
            "ec_uses_tensor_cores", "ec_launch_count", "ec_profile_enable", "ec_profile_read",
            "ec_route_static", "ec_route_static_bytes", "ec_shuffle", "ec_unshuffle",
-           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice", "ec_expert_gemm", "ec_validate_routing", "ec_debug_build"]
+           "ec_forward_only_workspace_bytes", "ec_capped_assignment", "ec_route_token_choice", "ec_expert_gemm", "ec_validate_routing", "ec_debug_build", "ec_backward_view"]
 EC_GEMM_XW1, EC_GEMM_HW2T, EC_GEMM_ATB = 0, 1, 2
 EC_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -41,6 +41,10 @@ class ec_config(C.Structure):
 class ec_saved_ptrs(C.Structure):
     _fields_ = [(name, C.c_void_p) for name in
                 ("S", "I", "G", "row_ptr", "slots", "X_in", "Z", "H", "X_e", "load", "requested")]
+
+
+class ec_backward_ptrs(C.Structure):
+    _fields_ = [(name, C.c_void_p) for name in ("dX_e", "dG", "dZ", "dX_in", "dL")] + [("dL_is_bf16", C.c_int32)]
 
 
 class EcError(RuntimeError):
@@ -72,6 +76,7 @@ def lib():
         L.ec_validate_routing.restype = C.c_int
         L.ec_validate_routing.argtypes = [P, V, V, V, C.POINTER(C.c_int64), V, C.c_size_t, V]
         L.ec_debug_build.restype = C.c_int; L.ec_debug_build.argtypes = []
+        L.ec_backward_view.restype = C.c_int; L.ec_backward_view.argtypes = [P, V, C.POINTER(ec_backward_ptrs)]
         L.ec_route_static.restype = C.c_int
         L.ec_route_static.argtypes = [P, V, V, V, V, V, V, V, V]
         L.ec_route_static_bytes.restype = C.c_size_t; L.ec_route_static_bytes.argtypes = [P]
@@ -329,6 +334,24 @@ def ec_profile_read(max_stages: int = 40):
     if cnt < 0:
         raise EcError(EC_ERR_CUDA, "ec_profile_read")
     return [(names[i].decode(), float(ms[i])) for i in range(cnt)]
+
+
+def backward_view(cfg, ws) -> dict:
+    """Torch views of the backward pass's intermediates in the workspace (no copies; valid until the workspace is used again)."""
+    v = ec_backward_ptrs()
+    _check(lib().ec_backward_view(C.byref(cfg), _ptr(ws), C.byref(v)), "ec_backward_view")
+    k, n, E, d, f = slots_per_expert(cfg), total_tokens(cfg), cfg.E, cfg.d_model, cfg.d_ff
+    dt, es, base = _torch_dtype(cfg), (4 if cfg.dtype == EC_F32 else 2), ws.data_ptr()
+
+    def view(addr, shape, dtype, esz):
+        cnt = 1
+        for s_ in shape:
+            cnt *= s_
+        return ws[addr - base:addr - base + cnt * esz].view(dtype).view(*shape)
+
+    dl = (torch.bfloat16, 2) if v.dL_is_bf16 else (torch.float32, 4)
+    return dict(dX_e=view(v.dX_e, (E, k, d), dt, es), dG=view(v.dG, (E, k), torch.float32, 4), dZ=view(v.dZ, (E, k, f), dt, es),
+                dX_in=view(v.dX_in, (E, k, d), dt, es), dL=view(v.dL, (n, E), *dl))
 
 
 def saved_view(cfg, saved) -> dict:

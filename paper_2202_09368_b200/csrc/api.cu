@@ -473,7 +473,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   tx.M = (int)D.n; tx.N = D.d; tx.K = D.E; tx.batches = 1;
   tx.epi = EPI_ADD_SLOTS; tx.C = dX; tx.ldc = D.d; tx.status = status;
   tx.row_ptr = row_ptr; tx.slots = slots; tx.rows = dX_in; tx.ld_rows = D.d; tx.slots_total = D.slots;
-  const bool tc_gate = D.dtype == EC_BF16 && tc_gemm_supported(tw) && tc_gemm_supported(tx);
+  const bool tc_gate = D.dtype == EC_BF16 && tc_gemm_supported(tw) && tc_gemm_supported(tx);     // mirrored by gate_grads_on_tc()
   EC_CUDA(launch_bwd_softmax(S, dG, row_ptr, slots, dL, tc_gate ? 1 : 0, D.n, D.E, D.k, status, st));
   prof_mark("bwd_softmax", st);
   if (tc_gate) {
@@ -544,6 +544,33 @@ ec_status ec_validate_routing(const ec_config* c, const int32_t* I, const int32_
   EC_CUDA(cudaMemcpyAsync(h, counters, sizeof(h), cudaMemcpyDeviceToHost, st));
   EC_CUDA(cudaStreamSynchronize(st));
   *violations = h[0];
+  return EC_OK;
+}
+
+namespace {
+// Whether ec_moe_backward runs dWg and dX on the tensor cores (dL is then bf16): the shape part of its decision, the
+// pointers being 256-byte aligned parts of the workspace and 16-byte aligned arguments.
+bool gate_grads_on_tc(const Dims& D) {
+  if (D.dtype != EC_BF16) return false;
+  const int P = dwg_splits(D);
+  const int64_t cut = (((D.n + P - 1) / P) + 63) / 64 * 64;
+  TcGemmArgs tw; memset(&tw, 0, sizeof(tw));
+  tw.A = tw.B = tw.C = (void*)256; tw.a_mn_major = 1; tw.lda = D.d; tw.b_mn_major = 1; tw.ldb = D.E;
+  tw.M = D.d; tw.N = D.E; tw.K = (int)cut; tw.batches = P; tw.k_split = 1; tw.k_total = D.n;
+  tw.epi = EPI_STORE; tw.c_f32 = 1; tw.ldc = D.E; tw.batch_c = (int64_t)D.d * D.E;
+  TcGemmArgs tx; memset(&tx, 0, sizeof(tx));
+  tx.A = tx.B = tx.C = (void*)256; tx.lda = D.E; tx.ldb = D.E; tx.M = (int)D.n; tx.N = D.d; tx.K = D.E; tx.batches = 1;
+  tx.epi = EPI_ADD_SLOTS; tx.ldc = D.d; tx.row_ptr = (const int32_t*)256; tx.slots = (const int32_t*)256; tx.rows = (void*)256; tx.ld_rows = D.d;
+  return tc_gemm_supported(tw) && tc_gemm_supported(tx);
+}
+}  // namespace
+
+ec_status ec_backward_view(const ec_config* c, void* ws, ec_backward_ptrs* out) {
+  Dims D; ec_status s = check_cfg(c, &D); if (s != EC_OK) return s;
+  if (!ws || !out) return EC_ERR_INVALID_ARG;
+  const WsLayout W = ws_layout(D); char* w = (char*)ws;
+  out->dX_e = w + W.dX_e; out->dG = (float*)(w + W.dG); out->dZ = w + W.dZ; out->dX_in = w + W.dX_in; out->dL = w + W.dL;
+  out->dL_is_bf16 = gate_grads_on_tc(D) ? 1 : 0;
   return EC_OK;
 }
 
