@@ -39,3 +39,15 @@ def test_random_shapes(dtype, groups, n, d, dff, E, c, k):
     li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=n + E)
     gelu = "tanh" if (n + d) % 5 == 0 else "erf"
     run_and_check(n, d, dff, E, c, dtype, li, gelu=gelu, groups=groups)
+
+
+@pytest.mark.parametrize("dtype,groups,n,d,dff,E,c,k", [t for t in _cases(40, seed=77) if t[5] >= 2][:16])
+def test_random_shapes_token_choice_and_biases(dtype, groups, n, d, dff, E, c, k):
+    """The same random shapes through the token-choice contrast routing (every second case) and with the bias terms of
+    Eq. 3 (two cases in three): empty slots, dropped requests, skipped tiles and bias gradients at odd sizes."""
+    token = (n + E) % 2 == 0
+    li = IN.make_layer_inputs(groups * n, d, dff, E, dtype, seed=n + E + 1, expert_skew=0.5 if token else 0.0)
+    biases = None
+    if (n + d) % 3 != 0:
+        biases = (IN.normal_tensor((E, dff), 0.5, n, IN.TID_AUX, dtype), IN.normal_tensor((E, d), 0.5, n + 1, IN.TID_AUX, dtype))
+    run_and_check(n, d, dff, E, c, dtype, li, groups=groups, router="token" if token else "expert", biases=biases)
