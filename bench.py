@@ -102,11 +102,13 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def workload_desc(name, groups=1, cap_b=0, cap_iters=100):
+def workload_desc(name, groups=1, cap_b=0, cap_iters=100, fuse_gather=False):
     n, d, dff, E, c = WORKLOADS[name]
     how = "one routing group per GPU" if groups == 1 else f"{groups} routing groups of {n // groups} tokens per GPU"
     if cap_b:
         how += f", at most {cap_b} experts per token ({cap_iters} solver rounds)"
+    if fuse_gather:
+        how += ", X_in read in place through I (fuse_gather)"
     return (f"{name}: n={n} d={d} d_ff={dff} E={E} c={c} k={int(n * c / E)} fwd+bwd, bf16 storage / fp32 accumulate, "
             f"{how}")
 
@@ -228,7 +230,7 @@ def run_reference(args):
            "n_gpus": args.gpus, "steps": ran, "steps_requested": args.steps, "warmup": 0, "ms_per_step": 1e3 * n / v,
            "ms_per_step_is": "extrapolated: the time of one whole step at the sampled rate, not the time the sample took",
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters)},
+           "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters, args.fuse_gather)},
            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": what},
            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
@@ -262,7 +264,8 @@ def run_gpu(args):
     n, d, dff, E, c = WORKLOADS[args.workload]
     bf = torch.bfloat16
     assert n % args.groups == 0
-    cfg = B.make_config(n // args.groups, d, dff, E, c, bf, groups=args.groups, cap_b=args.cap_b, cap_iters=args.cap_iters)
+    cfg = B.make_config(n // args.groups, d, dff, E, c, bf, groups=args.groups, cap_b=args.cap_b, cap_iters=args.cap_iters,
+                        fuse_gather=args.fuse_gather)
     seed = rank                                                   # each rank routes its own group
     chunk = 1 << 26
     X = IN.normal_tensor((n, d), 1.0, seed, IN.TID_X, bf, dev, chunk)
@@ -398,7 +401,7 @@ def run_gpu(args):
                         "sm_mhz": region_mhz, "median_ms": round(ms_step, 4), "best_ms": round(min(region_ms), 4),
                         "ms_x_mhz": [round(a * b, 1) if b else None for a, b in zip(region_ms, region_mhz)]},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters),
+            "config": {"workload": workload_desc(args.workload, args.groups, args.cap_b, args.cap_iters, args.fuse_gather),
                        "l2": "inputs larger than L2 (weights + activations per step >> 126 MB), no flush"
                              if args.workload != "small" else "small case, L2 resident",
                        "tensor_cores": bool(B.ec_uses_tensor_cores(cfg)),
@@ -415,6 +418,7 @@ def run_gpu(args):
                          "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": gemm_traffic(args.workload, E),
                          "flops_per_launch": fl["gemm"], "avg_launch_ms": gemm_avg_ms},
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
+            "saved_bytes": int(B.ec_saved_bytes(cfg)),
             "layer_tflops": (fl["fwd"] + fl["bwd"]) / (ms_step * 1e-3) / 1e12,
             "cpu_baseline": cpu,
         }
@@ -718,6 +722,7 @@ def main():
     ap.add_argument("--cap-b", type=int, default=0, help="at most this many experts per token (Section 3.3); 0 = plain expert choice")
     ap.add_argument("--cap-iters", type=int, default=100, help="rounds of the capped solver")
     ap.add_argument("--groups", type=int, default=1, help="route the n tokens as this many independent groups")
+    ap.add_argument("--fuse-gather", action="store_true", help="the expert GEMMs read the chosen rows of X in place; X_in is not written")
     ap.add_argument("--routing", action="store_true", help="routing-only stress grid instead of the layer benchmark")
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")

@@ -86,7 +86,12 @@ typedef struct {
   int32_t cap_iters; /* rounds of Dykstra's algorithm (the paper: at most 100), >= 1            */
   double cap_lambda; /* weight of the entropy term (the paper: 0.001), > 0                      */
   int32_t router;    /* ec_router; the token-choice contrast needs cap_b = 0 and E >= 2         */
-  int32_t reserved;  /* 0                                                                       */
+  /* 1: Eq. 3's shuffle X_in = P . X is never written.  GEMM-1 and the dW1 product read the chosen rows of X in place
+   * through I (row-indexed TMA loads on the tensor-core path), the blob of ec_saved_bytes is smaller by E*k*d elements
+   * and ec_saved_view reports X_in = NULL; every result is bit-identical to fuse_gather = 0.  It trades time for that
+   * memory: the rows are fetched again for every column tile, which is slower than gathering once.  Expert choice
+   * only (empty slots have no row to read).  0: the rows are gathered once into X_in.                               */
+  int32_t fuse_gather;
 } ec_config;
 
 /* Views into the forward->backward blob (device pointers), for inspection and tests. */

@@ -35,7 +35,7 @@ class ec_config(C.Structure):
     _fields_ = [("n", C.c_int64), ("d_model", C.c_int32), ("d_ff", C.c_int32), ("E", C.c_int32),
                 ("groups", C.c_int32), ("c", C.c_double), ("dtype", C.c_int32), ("gelu", C.c_int32),
                 ("cap_b", C.c_int32), ("cap_iters", C.c_int32), ("cap_lambda", C.c_double),
-                ("router", C.c_int32), ("reserved", C.c_int32)]
+                ("router", C.c_int32), ("fuse_gather", C.c_int32)]
 
 
 class ec_saved_ptrs(C.Structure):
@@ -103,13 +103,14 @@ def status_string(code: int) -> str:
 
 
 def make_config(n, d_model, d_ff, E, c, dtype=torch.float32, gelu="erf", groups=1, cap_b=0, cap_iters=100,
-                cap_lambda=1e-3, router="expert") -> ec_config:
+                cap_lambda=1e-3, router="expert", fuse_gather=False) -> ec_config:
     """cap_b > 0: at most cap_b experts per token (Section 3.3) with the paper's solver settings as defaults.
-    router = "token": the token-choice top-2 contrast of Section 3.1 with expert buffers of n*c/E slots."""
+    router = "token": the token-choice top-2 contrast of Section 3.1 with expert buffers of n*c/E slots.
+    fuse_gather: Eq. 3's X_in = P.X is read in place by the expert GEMMs instead of being written (smaller saved blob)."""
     dt = {torch.float32: EC_F32, torch.bfloat16: EC_BF16}[dtype]
     return ec_config(int(n), int(d_model), int(d_ff), int(E), int(groups), float(c), dt,
                      {"erf": EC_GELU_ERF, "tanh": EC_GELU_TANH}[gelu], int(cap_b), int(cap_iters), float(cap_lambda),
-                     {"expert": EC_ROUTER_EXPERT_CHOICE, "token": EC_ROUTER_TOKEN_TOP2}[router], 0)
+                     {"expert": EC_ROUTER_EXPERT_CHOICE, "token": EC_ROUTER_TOKEN_TOP2}[router], int(bool(fuse_gather)))
 
 
 def ec_capacity(cfg: ec_config) -> int:
@@ -377,6 +378,6 @@ def saved_view(cfg, saved) -> dict:
                      requested=view(v.requested, (cfg.groups, E), torch.int32, 4))
     return dict(**extra, S=view(v.S, (n, E), torch.float32, 4), I=view(v.I, (E, k), torch.int32, 4),
                 G=view(v.G, (E, k), torch.float32, 4), row_ptr=view(v.row_ptr, (n + 1,), torch.int32, 4),
-                slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es),
+                slots=view(v.slots, (E * k,), torch.int32, 4), X_in=view(v.X_in, (E, k, d), dt, es) if v.X_in else None,
                 Z=view(v.Z, (E, k, f), dt, es), H=view(v.H, (E, k, f), dt, es),
                 X_e=view(v.X_e, (E, k, d), torch.float32, 4))

@@ -19,7 +19,7 @@ inline size_t esize(int dtype) { return dtype == EC_F32 ? 4 : 2; }
 // n: all tokens of the call (groups * tokens per group), k: slots per expert (groups * k per group),
 // slots = E * k; ng, kg: the per-group values Eq. 1 is about.
 struct Dims { int64_t n, k, slots, ng, kg; int d, dff, E, groups; int dtype, gelu; size_t eb;
-              int cap_b, cap_iters; double cap_lambda; int router; };
+              int cap_b, cap_iters; double cap_lambda; int router, fuse; };
 
 ec_status check_cfg(const ec_config* c, Dims* D) {
   if (!c) return EC_ERR_INVALID_ARG;
@@ -41,7 +41,9 @@ ec_status check_cfg(const ec_config* c, Dims* D) {
   }
   if (c->router != EC_ROUTER_EXPERT_CHOICE && c->router != EC_ROUTER_TOKEN_TOP2) return EC_ERR_INVALID_ARG;
   if (c->router == EC_ROUTER_TOKEN_TOP2 && (c->cap_b != 0 || c->E < 2)) return EC_ERR_INVALID_ARG;
-  if (D) { D->router = c->router; D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
+  if (c->fuse_gather != 0 && c->fuse_gather != 1) return EC_ERR_INVALID_ARG;
+  if (c->fuse_gather && c->router != EC_ROUTER_EXPERT_CHOICE) return EC_ERR_INVALID_ARG;   // empty slots have no row of X to read
+  if (D) { D->router = c->router; D->fuse = c->fuse_gather; D->ng = c->n; D->kg = k; D->groups = c->groups; D->n = c->n * c->groups; D->k = k * c->groups;
            D->slots = (int64_t)c->E * D->k; D->d = c->d_model; D->dff = c->d_ff;
            D->E = c->E; D->dtype = c->dtype; D->gelu = c->gelu; D->eb = eb;
            D->cap_b = c->cap_b; D->cap_iters = c->cap_iters; D->cap_lambda = c->cap_lambda; }
@@ -58,7 +60,7 @@ SavedLayout saved_layout(const Dims& D, bool with_z = true) {
   L.G = take((size_t)D.slots * 4);
   L.row_ptr = take((size_t)(D.n + 1) * 4);
   L.slots = take((size_t)D.slots * 4);
-  L.X_in = take((size_t)D.slots * D.d * D.eb);
+  L.X_in = take(D.fuse ? 0 : (size_t)D.slots * D.d * D.eb);       // with fuse_gather the rows of X are read in place
   L.Z = take(with_z ? (size_t)D.slots * D.dff * D.eb : 0);
   L.H = take((size_t)D.slots * D.dff * D.eb);
   L.X_e = take((size_t)D.slots * D.d * 4);          // fp32 on both paths
@@ -147,6 +149,9 @@ struct BatchedGemm {
   int c_f32;                                         // C is fp32 regardless of the path's dtype
   const int32_t* batch_rows; int ragged;             // see TcGemmArgs: meaningful rows per batch along M (1) or K (2)
   const void* bias;                                  // [batches, N] of the path's dtype, added to the accumulator (Eq. 3's omitted bias terms)
+  // A's stored rows are rows of the matrix at A (a_rows_total rows, pitch lda) picked through a_rows (Eq. 3's
+  // X_in = P . X read in place): row r of batch b is matrix row a_rows[b * a_rows_batch + r]
+  const int32_t* a_rows; int64_t a_rows_batch, a_rows_total;
 };
 
 ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaStream_t st) {
@@ -158,6 +163,7 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
     t.epi = b.epi; t.gelu = D.gelu; t.C = b.C; t.C2 = b.C2; t.Zin = b.Zin; t.ldc = b.ldc; t.batch_c = b.batch_c; t.c_f32 = b.c_f32;
     t.status = status_word;
     t.batch_rows = b.batch_rows; t.ragged = b.ragged; t.bias = b.bias;
+    t.a_rows = b.a_rows; t.a_rows_batch = b.a_rows_batch; t.a_rows_total = b.a_rows_total;
     if (tc_gemm_supported(t)) { EC_CUDA(launch_gemm_tc(t, st)); return EC_OK; }
   }
   GemmArgs g; memset(&g, 0, sizeof(g));
@@ -169,6 +175,8 @@ ec_status run_gemm(const Dims& D, const BatchedGemm& b, int* status_word, cudaSt
   g.ldc = b.ldc; g.batch_a = b.batch_a; g.batch_b = b.batch_b; g.batch_c = b.batch_c;
   g.epi = b.epi; g.gelu = D.gelu; g.C2 = b.C2; g.Zin = b.Zin;
   g.bias = b.bias; g.bias_dtype = D.dtype;
+  g.a_rows = b.a_rows; g.a_rows_batch = b.a_rows_batch; g.a_rows_total = b.a_rows_total; g.a_rows_k = b.a_mn;   // the stored rows of A run along K when it is MN-major
+  g.status = status_word;
   EC_CUDA(launch_gemm_simt(g, st));
   return EC_OK;
 }
@@ -272,7 +280,7 @@ ec_status ec_saved_view(const ec_config* c, void* saved, ec_saved_ptrs* out) {
   const SavedLayout L = saved_layout(D); char* b = (char*)saved;
   out->S = (float*)(b + L.S); out->I = (int32_t*)(b + L.I); out->G = (float*)(b + L.G);
   out->row_ptr = (int32_t*)(b + L.row_ptr); out->slots = (int32_t*)(b + L.slots);
-  out->X_in = b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = (float*)(b + L.X_e);
+  out->X_in = D.fuse ? nullptr : b + L.X_in; out->Z = b + L.Z; out->H = b + L.H; out->X_e = (float*)(b + L.X_e);
   out->load = D.router ? (int32_t*)(b + L.load) : nullptr;
   out->requested = D.router ? (int32_t*)(b + L.requested) : nullptr;
   return EC_OK;
@@ -398,11 +406,14 @@ ec_status ec_moe_forward(const ec_config* c, const void* X, const void* Wg, cons
   int32_t* requested = D.router ? (int32_t*)(sv + L.requested) : nullptr;
   const int32_t* rag = D.router && D.groups == 1 ? load : nullptr;
   if ((s = route_impl(D, X, Wg, S, I, G, row_ptr, slots, w, W, st, load, requested)) != EC_OK) return s;
-  EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, D.n, status, st));
-  prof_mark("gather", st);
+  if (!D.fuse) {
+    EC_CUDA(launch_gather(D.dtype, X, I, X_in, D.slots, D.d, D.n, status, st));
+    prof_mark("gather", st);
+  }
   const int64_t kd = D.k * D.d, kf = D.k * D.dff, df = (int64_t)D.d * D.dff;
-  // Z = X_in[i] . W1[i],  H = GeLU(Z)
+  // Z = X_in[i] . W1[i],  H = GeLU(Z); with fuse_gather X_in[i] is rows I[i, :] of X read in place
   BatchedGemm g1 = {X_in, 0, D.d, kd, W1, 1, D.dff, df, Z, D.dff, kf, (int)D.k, D.dff, D.d, D.E, EPI_GELU, H, nullptr, 0, rag, 1, b1};
+  if (D.fuse) { g1.A = X; g1.batch_a = 0; g1.a_rows = I; g1.a_rows_batch = D.k; g1.a_rows_total = D.n; }
   if ((s = run_gemm(D, g1, status, st)) != EC_OK) return s;
   prof_mark("gemm1_gelu", st);
   // X_e = H[i] . W2[i]^T, kept in fp32
@@ -455,6 +466,7 @@ ec_status ec_moe_backward(const ec_config* c, const void* X, const void* Wg, con
   prof_mark("gemm_dW2", st);
   // dW1[i] = X_in[i]^T . dZ[i]
   BatchedGemm g5 = {X_in, 1, D.d, kd, dZ, 1, D.dff, kf, dW1, D.dff, df, D.d, D.dff, (int)D.k, D.E, EPI_STORE, nullptr, nullptr, 0, rag, 2, nullptr};
+  if (D.fuse) { g5.A = X; g5.batch_a = 0; g5.a_rows = I; g5.a_rows_batch = D.k; g5.a_rows_total = D.n; }   // X_in[i] again read from X through I
   if ((s = run_gemm(D, g5, status, st)) != EC_OK) return s;
   prof_mark("gemm_dW1", st);
   // dX_in[i] = dZ[i] . W1[i]^T

@@ -33,7 +33,8 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
   const int b = blockIdx.z;
-  const TA* A = (const TA*)g.A + (int64_t)b * g.batch_a;
+  const TA* A = (const TA*)g.A + (g.a_rows ? 0 : (int64_t)b * g.batch_a);
+  const int32_t* arow = g.a_rows ? g.a_rows + (int64_t)b * g.a_rows_batch : nullptr;
   const TB* B = (const TB*)g.B + (int64_t)b * g.batch_b;
   const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;     // row tiles on grid.x: M (tokens) is the dimension without a limit
   const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
@@ -51,7 +52,19 @@ __global__ void __launch_bounds__(NT) gemm_simt_kernel(GemmArgs g) {
       const int idx = tid + r * NT;
       const int mm = a_k_fast ? idx / BK : idx % BM, kk = a_k_fast ? idx % BK : idx / BM;
       const int m = m0 + mm, k = k0 + kk;
-      As[kk][mm] = (m < g.M && k < Kb) ? ldv(A, (int64_t)m * g.sam + (int64_t)k * g.sak) : 0.f;
+      float av = 0.f;
+      if (m < g.M && k < Kb) {
+        // with a row selection the index along M (or along K) goes through the list first
+        int64_t mi = m, ki = k;
+        bool ok = true;
+        if (arow) {
+          const int sel = arow[g.a_rows_k ? k : m];
+          ok = idx_ok(sel, 0, g.a_rows_total, g.status);
+          if (g.a_rows_k) ki = sel; else mi = sel;
+        }
+        if (ok) av = ldv(A, mi * g.sam + ki * g.sak);
+      }
+      As[kk][mm] = av;
     }
 #pragma unroll
     for (int r = 0; r < BN * BK / NT; ++r) {

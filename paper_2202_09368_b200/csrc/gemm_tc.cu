@@ -92,6 +92,7 @@ struct TcParams {
   int64_t slots_total;                               // rows of `rows`: what the debug build checks the slot ids against
   const int32_t* batch_rows; int ragged;             // meaningful rows per batch along M (1) or K (2), zeros beyond
   const bf16* bias;                                  // EPI_GELU, EPI_STORE_F32: bias[b * N + n] joins every row of the accumulator
+  const int32_t* a_rows; int64_t a_rows_batch; int a_rows_total;   // A's stored rows come from one matrix through this index list (tmA is then 2-D)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -156,6 +157,16 @@ __device__ __forceinline__ bool half_all(int half, bool ok) {          // true w
   asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %2, 0;\n barrier.cta.red.and.pred q, %1, 128, p;\n selp.u32 %0, 1, 0, q;\n}\n"
                : "=r"(r) : "r"(1 + half), "r"((uint32_t)ok) : "memory");
   return r != 0;
+}
+// Row-indexed loads (tile::gather4): four rows of a 2-D tensor, chosen by index, 64 elements (128 bytes) of each
+// starting at column c0, land as four consecutive 128-byte rows at dst.  The tensor map's box is one row high.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int r0, int r1, int r2, int r3) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
+__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int r0, int r1, int r2, int r3) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+               ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -353,6 +364,70 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (gave_up) {
     // nothing: fall through to the exit sequence
+  } else if (warp == 0 && p.a_rows != nullptr) {
+    // ------------------------------------------------------------------ TMA producer, A rows chosen through an index list
+    // Eq. 3's X_in = P . X is not written: the stage's 128 x 64 block of A is filled by 32 row-indexed loads of four
+    // rows each, one per lane (K-major A: the tile's 128 rows of M, the same for every k-block; MN-major A: two
+    // 64-wide blocks of M times the k-block's 64 rows of K).  The shared-memory image is the one a box load of
+    // X_in would have left (the 128-byte swizzle is a function of the shared-memory address).  Positions past the
+    // end of the batch's list take its last entry: such rows of A meet either rows of C that are clipped (M) or
+    // rows of B that the TMA unit zero-fills (K).  Lane 0 also loads B and announces the bytes, as the plain producer.
+    int stage = 0; uint32_t phase = 0;
+    const uint32_t leader_full0 = CTAS == 2 ? map_to_cta(full0, 0) : full0;
+    const int nidx = p.a_mn ? p.K : p.M;               // stored rows of A per batch
+    auto pick = [&](const int32_t* list, int pos) {
+      const int r = __ldg(list + min(pos, nidx - 1));
+      return idx_ok(r, 0, p.a_rows_total, p.status) ? r : 0;
+    };
+    for (int tile = first_tile; tile < p.total_tiles && !gave_up; tile += tile_step) {
+      const int b = tile / (p.tiles_m * p.tiles_n);
+      const int mt = p.n_fast ? (tile / p.tiles_n) % p.tiles_m : tile % p.tiles_m;
+      const int nt = p.n_fast ? tile % p.tiles_n : (tile / p.tiles_m) % p.tiles_n;
+      const int m0 = mt * TM + (int)rank * BM, n0 = nt * BN + (int)rank * kBHalf;
+      const int32_t* rows_b = p.a_rows + (int64_t)b * p.a_rows_batch;
+      int ri[4];
+      const int rbase = p.a_mn ? 4 * (lane & 15) : m0 + 4 * lane;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) ri[j] = pick(rows_b, rbase + j);
+      for (int kb = 0; kb < p.kblocks; ++kb) {
+        const bool ok = mbar_wait(empty0 + 8 * stage, phase ^ 1, abort_flag, p.status, 1);
+        if (!__all_sync(0xffffffffu, ok)) { gave_up = true; break; }
+        const uint32_t sa = smem_base + stage * kStage, sb = sa + kABytes;
+        const int k0 = kb * BK;
+        const uint32_t bar = (CTAS == 2 ? leader_full0 : full0) + 8 * stage;
+        if (lane == 0) {
+          if constexpr (CTAS == 2) {
+            if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * kStage);
+            if (p.b_mn) {
+#pragma unroll
+              for (int j = 0; j < BNL / 64; ++j)
+                tma_load_3d_pair(sb + j * (BK * 128), &tmB, bar, n0 + (64 * j / kBHalf) * kMmaN + 64 * j % kBHalf, k0, b);
+            } else {
+#pragma unroll
+              for (int j = 0; j < BNL / kBHalf; ++j) tma_load_3d_pair(sb + j * (kBHalf * 128), &tmB, bar, k0, n0 + j * kMmaN, b);
+            }
+          } else {
+            mbar_expect_tx(bar, kStage);
+            if (p.b_mn) {
+#pragma unroll
+              for (int j = 0; j < BNL / 64; ++j) tma_load_3d(sb + j * (BK * 128), &tmB, bar, n0 + 64 * j, k0, b);
+            } else {
+              tma_load_3d(sb, &tmB, bar, k0, n0, b);
+            }
+          }
+        }
+        __syncwarp();                                    // the announcement is made before any of the warp's copies can land
+        const uint32_t dst = p.a_mn ? sa + (lane >> 4) * (BK * 128) + (lane & 15) * 512 : sa + lane * 512;
+        const int col = p.a_mn ? m0 + 64 * (lane >> 4) : k0;
+        if constexpr (CTAS == 2) tma_gather4_pair(dst, &tmA, bar, col, ri[0], ri[1], ri[2], ri[3]);
+        else tma_gather4(dst, &tmA, bar, col, ri[0], ri[1], ri[2], ri[3]);
+        if (p.a_mn && kb + 1 < p.kblocks) {              // the next k-block's rows of K, fetched while this one lands
+#pragma unroll
+          for (int j = 0; j < 4; ++j) ri[j] = pick(rows_b, (kb + 1) * BK + rbase + j);
+        }
+        if (++stage == S) { stage = 0; phase ^= 1; }
+      }
+    }
   } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -791,6 +866,20 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, in
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map for row-indexed loads (tile::gather4) from a matrix [rows][inner] with row pitch ld: two dimensions,
+// a box of 64 elements of one row.
+bool make_gather_map(CUtensorMap* tm, const void* base, int64_t inner, int64_t rows, int64_t ld) {
+  auto enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64, 1};
+  cuuint32_t es[2] = {1, 1};
+  return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 512 columns per tile for a CTA pair on a long contraction with a plain store; else 256 columns when the
 // tile is a CTA pair's; a single CTA (M <= 128: few rows per expert, the product
 // streams the weights) does better with 128, whose smaller stages leave room for five of them instead of three
@@ -878,6 +967,7 @@ bool tc_gemm_supported(const TcGemmArgs& g) {
   if ((int64_t)g.lda * 2 >= ((int64_t)1 << 40) || (int64_t)g.ldb * 2 >= ((int64_t)1 << 40)) return false;
   if (g.batch_rows && (g.k_split || (g.ragged != 1 && g.ragged != 2))) return false;
   if (g.bias && (((uintptr_t)g.bias & 15) || g.k_split || !(g.epi == EPI_GELU || (g.epi == EPI_STORE && g.c_f32)))) return false;
+  if (g.a_rows && (g.k_split || g.batch_rows || g.epi == EPI_SOFTMAX || g.a_rows_total < 1 || g.a_rows_total >= ((int64_t)1 << 31))) return false;
   return true;
 }
 
@@ -893,7 +983,8 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   // operand maps: with k_split both are single matrices whose K extent is the whole contraction
   const int64_t kext = g.k_split ? g.k_total : g.K;
   const int64_t ob = g.k_split ? 1 : g.batches;
-  const bool oka = g.a_mn_major ? make_map(&ta, g.A, g.M, kext, ob, g.lda, g.batch_a, 64, BK)
+  const bool oka = g.a_rows ? make_gather_map(&ta, g.A, g.a_mn_major ? g.M : g.K, g.a_rows_total, g.lda)
+                 : g.a_mn_major ? make_map(&ta, g.A, g.M, kext, ob, g.lda, g.batch_a, 64, BK)
                                 : make_map(&ta, g.A, kext, g.M, ob, g.lda, g.batch_a, BK, BM);
   const bool okb = g.b_mn_major ? make_map(&tb, g.B, g.N, kext, ob, g.ldb, g.batch_b, 64, BK)
                                 : make_map(&tb, g.B, kext, g.N, ob, g.ldb, g.batch_b, BK, bnl > 128 ? 128 : bnl);
@@ -925,6 +1016,7 @@ cudaError_t launch_gemm_tc(const TcGemmArgs& g, cudaStream_t st) {
   p.row_ptr = g.row_ptr; p.slots = g.slots; p.rows = (const bf16*)g.rows; p.ld_rows = g.ld_rows; p.slots_total = g.slots_total;
   p.batch_rows = g.batch_rows; p.ragged = g.ragged;
   p.bias = (const bf16*)g.bias;
+  p.a_rows = g.a_rows; p.a_rows_batch = g.a_rows_batch; p.a_rows_total = (int)g.a_rows_total;
   switch (g.epi) {
     case EPI_STORE: return g.c_f32 ? launch_bn<EPI_STORE_F32>(bn, ctas, ta, tb, tc, tc2, p, st)
                                    : launch_bn<EPI_STORE>(bn, ctas, ta, tb, tc, tc2, p, st);

@@ -118,6 +118,10 @@ struct GemmArgs {
   const int32_t* row_ptr; const int32_t* slots; const void* rows; int64_t ld_rows;  // EPI_ADD_SLOTS
   int64_t slots_total; int* status;    // EPI_ADD_SLOTS, debug build: range of the slot ids and where a bad one is recorded
   const void* bias; int bias_dtype;    // not null: bias[b * N + n] is added to the accumulator before the epilogue's function
+  // a_rows != null: A is a row selection of one matrix (Eq. 3's X_in = P . X without the copy).  The index along M
+  // (a_rows_k = 0) or along K (a_rows_k = 1) is replaced by a_rows[b * a_rows_batch + index], which must lie in
+  // [0, a_rows_total); batch_a is unused.
+  const int32_t* a_rows; int64_t a_rows_batch, a_rows_total; int a_rows_k;
 };
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t st);
 
@@ -152,6 +156,11 @@ struct TcGemmArgs {
   // bias != null (EPI_GELU, or EPI_STORE with fp32 C): bf16 bias[b * N + n] is added to every row of the accumulator
   // before the epilogue's function (the bias terms Eq. 3 leaves out); 16-byte aligned.
   const void* bias;
+  // a_rows != null: the shuffle of Eq. 3 read in place.  A's stored rows (its M rows when K-major, its K rows when
+  // MN-major) are rows of ONE matrix [a_rows_total, lda] at A, chosen through an index list: stored row r of batch b
+  // is matrix row a_rows[b * a_rows_batch + r] (every entry in [0, a_rows_total)).  batch_a is unused; not with
+  // k_split or batch_rows.
+  const int32_t* a_rows; int64_t a_rows_batch, a_rows_total;
 };
 constexpr int EPI_SOFTMAX = 4;
 bool tc_gemm_supported(const TcGemmArgs& g);

@@ -141,7 +141,8 @@ def run_and_check(n, d, dff, E, c, dtype, li, gelu="erf", backward=True, check_S
         check_routing(cfg, v["S"], v["I"], v["G"], v["row_ptr"], v["slots"])
     f = O.forward(Xn, Wgn, W1n, W2n, c, gelu, S_override=to_np(v["S"]), I_override=v["I"].cpu().numpy(), groups=groups,
                   router=router, b1=b1n, b2=b2n)
-    assert np.array_equal(v["X_in"].float().cpu().numpy(), f["X_in"].astype(np.float32))    # the shuffle of Eq. 3 is a copy
+    if v["X_in"] is not None:                      # with fuse_gather the shuffle of Eq. 3 is never written
+        assert np.array_equal(v["X_in"].float().cpu().numpy(), f["X_in"].astype(np.float32))    # it is a copy
     filled = v["I"].cpu().numpy() >= 0             # all slots with expert choice; token choice leaves some empty, and
     got = {}                                       # what the library keeps for an empty slot is unspecified
     for name in ("Z", "H", "X_e"):

@@ -70,9 +70,10 @@ def test_validate_routing_accepts_what_the_router_makes_and_counts_what_is_wrong
 
 
 @pytest.mark.parametrize("dtype,n,d,dff,E,c,router", [(F32, 300, 36, 100, 3, 1.5, "expert"), (BF16, 1024, 128, 256, 8, 2.0, "expert"),
-                                                      (BF16, 2048, 128, 384, 4, 2.6, "token"), (BF16, 1024, 128, 256, 8, 2.0, "capped")])
+                                                      (BF16, 2048, 128, 384, 4, 2.6, "token"), (BF16, 1024, 128, 256, 8, 2.0, "capped"),
+                                                      (BF16, 1024, 128, 256, 8, 2.0, "fused"), (F32, 300, 36, 100, 3, 1.5, "fused")])
 def test_debug_build_gives_the_same_bits_and_reports_nothing_on_valid_inputs(D, dtype, n, d, dff, E, c, router):
-    cap = dict(cap_b=3, cap_iters=20) if router == "capped" else {}
+    cap = dict(cap_b=3, cap_iters=20) if router == "capped" else dict(fuse_gather=True) if router == "fused" else {}
     rt = "token" if router == "token" else "expert"
     li = IN.make_layer_inputs(n, d, dff, E, dtype, seed=33, expert_skew=1.0 if rt == "token" else 0.0)
     X, Wg, W1, W2, dY = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2, li.dX_out))
@@ -89,14 +90,15 @@ def test_debug_build_gives_the_same_bits_and_reports_nothing_on_valid_inputs(D, 
         assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
 
 
+@pytest.mark.parametrize("fuse", [False, True])
 @pytest.mark.parametrize("dtype", [F32, BF16])
-def test_debug_build_survives_and_reports_corrupted_indices(D, dtype):
+def test_debug_build_survives_and_reports_corrupted_indices(D, dtype, fuse):
     """Only the debug library is given these: indices far outside their ranges in the saved blob between forward and
     backward, and in the arguments of the stand-alone shuffle and unshuffle.  Every bad access is skipped."""
     n, d, dff, E, c = 1024, 128, 256, 8, 2.0
     li = IN.make_layer_inputs(n, d, dff, E, dtype, seed=35)
     X, Wg, W1, W2, dY = (t.cuda() for t in (li.X, li.Wg, li.W1, li.W2, li.dX_out))
-    cfg = D.make_config(n, d, dff, E, c, dtype)
+    cfg = D.make_config(n, d, dff, E, c, dtype, fuse_gather=fuse)    # fused: the dW1 product reads rows of X through the bad I
     k = D.ec_capacity(cfg)
     ws = D.alloc_workspace(cfg)
     Y, saved = D.ec_moe_forward(cfg, X, Wg, W1, W2, ws=ws)

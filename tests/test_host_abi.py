@@ -54,6 +54,21 @@ def test_sizes_and_rejections():
     assert B.status_string(B.EC_ERR_TIMEOUT).startswith("a bounded")
 
 
+def test_fuse_gather_config():
+    """fuse_gather leaves X_in out of the blob and of the forward-only scratch, and is refused where slots can be empty."""
+    for dt, es in ((torch.float32, 4), (torch.bfloat16, 2)):
+        plain, fused = (B.make_config(256, 64, 256, 4, 2.0, dt, groups=2, fuse_gather=f) for f in (False, True))
+        x_in = 4 * 2 * 128 * 64 * es
+        assert x_in <= B.ec_saved_bytes(plain) - B.ec_saved_bytes(fused) < x_in + 256
+        fwd = lambda cfg: int(B.lib().ec_forward_only_workspace_bytes(ctypes.byref(cfg)))
+        assert x_in <= fwd(plain) - fwd(fused) < x_in + 256
+        assert B.ec_workspace_bytes(fused) == B.ec_workspace_bytes(plain)
+    assert B.ec_saved_bytes(B.make_config(256, 64, 256, 4, 2.0, router="token", fuse_gather=True)) == 0
+    bad = B.make_config(256, 64, 256, 4, 2.0)
+    bad.fuse_gather = 2
+    assert B.ec_saved_bytes(bad) == 0 and B.ec_workspace_bytes(bad) == 0
+
+
 def test_null_pointers_are_rejected_without_a_gpu():
     cfg = B.make_config(256, 64, 256, 4, 2.0)
     L = B.lib()
