@@ -98,8 +98,16 @@ class ClockSampler:
             except Exception:
                 pass
         sm.sort()
+        watts = []
+        for r in self.rows:
+            try:
+                watts.append(float(r[2]))
+            except Exception:
+                pass
+        # samples taken under load: the sampler also sees the moments before the first and after the last launch
+        watts = sorted(w for w in watts if w >= 0.8 * max(watts))
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx or None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "watts": watts[len(watts) // 2] if watts else None}
 
 
 def workload_desc(name, groups=1, cap_b=0, cap_iters=100, fuse_gather=False):
@@ -420,6 +428,11 @@ def run_gpu(args):
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
             "saved_bytes": int(B.ec_saved_bytes(cfg)),
             "layer_tflops": (fl["fwd"] + fl["bwd"]) / (ms_step * 1e-3) / 1e12,
+            # under the board's power cap a step costs what it costs in energy: watts (median of the samples taken
+            # under load) x time per step; per flop of the layer it compares with the vendor's large square product
+            # (`--gemms --loop-seconds`)
+            "energy": (lambda w: {"watts": w, "joules_per_step": round(w * ms_step * 1e-3, 3),
+                                  "pj_per_flop": round(w * ms_step * 1e-3 / (fl["fwd"] + fl["bwd"]) * 1e12, 4)} if w else None)(clocks.summary()["watts"]),
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
@@ -615,20 +628,50 @@ def run_gemms(args):
              ("dW = A^T . B", B.EC_GEMM_ATB, A, H, lambda o: torch.bmm(A.transpose(1, 2), H, out=o))]
     reps = max(10, args.steps)
     res = {}
+
+    def timed(fn, count):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(count):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / count
+
+    if args.loop_seconds > 0:
+        # Energy view: every product loops for --loop-seconds, long enough for the power controller to settle and for
+        # nvidia-smi to sample power and clocks; energy per flop = median watts x time per call / flops.  A large square
+        # product of the vendor library (nothing but tensor-core work, hardly any HBM traffic) calibrates the scale.
+        side = 8192
+        Sa, Sb, Sc = (torch.randn(side, side, device=dev, dtype=bf) for _ in range(3))
+        loops = [("square 8192^3", "torch_mm", lambda: torch.mm(Sa, Sb, out=Sc), 2.0 * side ** 3)]
+        for name, kind, a, b_, vendor in cases:
+            loops.append((name, "this_library", (lambda kind=kind, a=a, b_=b_: B.ec_expert_gemm(cfg, kind, a, b_, outs[kind], ws)), flops))
+            loops.append((name, "torch_bmm", (lambda kind=kind, vendor=vendor: vendor(outs[kind])), flops))
+        for name, tag, fn, fl in loops:
+            for _ in range(5):
+                fn()
+            count = max(20, int(args.loop_seconds * 1e3 / timed(fn, 10)))
+            with ClockSampler(torch.cuda.current_device()) as cs:
+                ms = timed(fn, count)
+            c = cs.summary()
+            res.setdefault(name, {})[tag] = {"tflops": round(fl / ms / 1e9, 1), "ms": round(ms, 4), "sm_mhz": c["sm_mhz"], "watts": c["watts"],
+                                             "pj_per_flop": round(c["watts"] * ms * 1e-3 / fl * 1e12, 4) if c["watts"] else None,
+                                             "reasons": c["reasons"]}
+            time.sleep(0.5)
+        assert B.ec_read_status(ws) == B.EC_OK
+        print(json.dumps({"metric": "expert_gemm_alone_energy", "unit": "each product alone in a loop of --loop-seconds; pJ per flop = watts x time / flops",
+                          "config": {"workload": f"{Eb} experts of {args.workload}: k={k} d={d} d_ff={dff}, bf16", "loop_seconds": args.loop_seconds},
+                          "cases": res}))
+        return
     for rnd in range(max(2, min(args.repeats, 3))):
         for name, kind, a, b_, vendor in cases:
             o = outs[kind]
             for tag, fn in (("this_library", lambda: B.ec_expert_gemm(cfg, kind, a, b_, o, ws)), ("torch_bmm", lambda: vendor(o))):
                 for _ in range(5):
                     fn()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                e0.record()
-                for _ in range(reps):
-                    fn()
-                e1.record()
-                torch.cuda.synchronize()
-                res.setdefault(name, {}).setdefault(tag, []).append(round(flops / (e0.elapsed_time(e1) / reps) / 1e9, 1))
+                res.setdefault(name, {}).setdefault(tag, []).append(round(flops / timed(fn, reps) / 1e9, 1))
     assert B.ec_read_status(ws) == B.EC_OK
     print(json.dumps({"metric": "expert_gemm_alone_tflops", "unit": "TFLOP/s, each product alone in a loop, rounds in order",
                       "config": {"workload": f"{Eb} experts of {args.workload}: k={k} d={d} d_ff={dff}, bf16", "calls_per_timing": reps},
@@ -727,6 +770,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="capacity-factor sweep of the forward pass instead of the layer benchmark")
     ap.add_argument("--route-case", default="", help="with --routing: one case 'n,E' or 'n,E,d' instead of the grid")
     ap.add_argument("--gemms", action="store_true", help="the expert GEMMs alone in a loop, torch.bmm beside them (calibration)")
+    ap.add_argument("--loop-seconds", type=float, default=0.0, help="with --gemms: loop every product this long and report watts, clocks and pJ per flop")
     ap.add_argument("--contrast", action="store_true", help="expert choice beside token-choice top-2 routing on identical inputs")
     ap.add_argument("--expert-skew", type=float, default=0.05, help="with --contrast: popularity offset of the experts' gate logits")
     args = ap.parse_args()
