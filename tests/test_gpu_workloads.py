@@ -100,6 +100,11 @@ def test_routing_groups_match_separate_calls():
     (2, 32768, 64, 2.0, BF16),                  # groups above the single-CTA size: histogram passes, k = 1024 per group
     (3, 20000, 8, 2.0, torch.float32),          # k = 5000 per group: candidates merged globally, multi-kernel sort
     (2, 17000, 12, 0.7, torch.float32),         # ragged k, E a multiple of 4 only
+    # bf16: the gate's softmax epilogue counts the selection's first histogram; groups that do not end on a warp's
+    # 32 rows, padded columns of a 64-wide tile, and the two-CTA tile whose warps split the columns of a row
+    (3, 20000, 8, 2.0, BF16),
+    (2, 17000, 40, 0.7, BF16),
+    (2, 40000, 136, 1.5, BF16),
 ])
 def test_routing_groups_large_groups(groups, n, E, c, dtype):
     """Routing groups on the multi-kernel top-k path (more than 16384 tokens per group)."""
@@ -115,10 +120,11 @@ def test_routing_groups_with_ties_on_the_multi_kernel_path():
     """Few distinct logits and large groups: thousands of exactly equal scores at the threshold of every expert
     and group, resolved toward the lower token by the walk in token order."""
     groups, n, d, E = 2, 20000, 16, 8
-    X, Wg = IN.quantised_gate_inputs(groups * n, d, E, 2, torch.float32)
-    cfg = B.make_config(n, d, 16, E, 2.0, torch.float32, groups=groups)
-    r = B.ec_route(cfg, X.cuda(), Wg.cuda())
-    check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
+    for dtype in (torch.float32, BF16):           # bf16: first histogram counted by the gate's epilogue
+        X, Wg = IN.quantised_gate_inputs(groups * n, d, E, 2, dtype)
+        cfg = B.make_config(n, d, 16, E, 2.0, dtype, groups=groups)
+        r = B.ec_route(cfg, X.cuda(), Wg.cuda())
+        check_routing(cfg, r.S, r.I, r.G, r.row_ptr, r.slots)
 
 
 @pytest.mark.parametrize("n,E,c,b,iters,lam,groups", [
