@@ -101,7 +101,7 @@ typedef struct {
   float* G;         /* [E, k]     gate weight of each slot, G[i,j] = S[I[i,j], i]      */
   int32_t* row_ptr; /* [n+1]      token -> range in `slots`                            */
   int32_t* slots;   /* [E*k]      flat slot ids of each token, ascending               */
-  void* X_in;       /* [E, k, d]  gathered expert inputs (Eq. 3)                       */
+  void* X_in;       /* [E, k, d]  gathered expert inputs (Eq. 3); NULL with fuse_gather  */
   void* Z;          /* [E, k, d'] X_in[i] . W1[i]                                      */
   void* H;          /* [E, k, d'] GeLU(Z)                                              */
   float* X_e;       /* [E, k, d]  expert outputs H[i] . W2[i]^T, fp32 on both paths    */
