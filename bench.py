@@ -63,12 +63,21 @@ class ClockSampler:
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
+    INSTANT = None                      # whether this driver's nvidia-smi knows power.draw.instant (asked once)
+
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        if ClockSampler.INSTANT is None:
+            try:
+                ClockSampler.INSTANT = subprocess.run(["nvidia-smi", "--query-gpu=power.draw.instant", "--format=csv,noheader,nounits",
+                                                       "-i", str(index)], capture_output=True, timeout=20).returncode == 0
+            except Exception:
+                ClockSampler.INSTANT = False
 
     def __enter__(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+            q = self.Q + (",power.draw.instant" if ClockSampler.INSTANT else "")      # an eighth column: the unaveraged reading
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
                                           "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -98,16 +107,23 @@ class ClockSampler:
             except Exception:
                 pass
         sm.sort()
-        watts = []
-        for r in self.rows:
-            try:
-                watts.append(float(r[2]))
-            except Exception:
-                pass
-        # samples taken under load: the sampler also sees the moments before the first and after the last launch
-        watts = sorted(w for w in watts if w >= 0.8 * max(watts))
+        def under_load(col):
+            # samples taken under load: the sampler also sees the moments before the first and after the last launch
+            w = []
+            for r in self.rows:
+                try:
+                    w.append(float(r[col]))
+                except Exception:
+                    pass
+            if not w:
+                return None
+            w = [x for x in w if x >= 0.8 * max(w)]
+            return round(sum(w) / len(w), 1)
+        # power.draw is the driver's running average (right for loops of seconds, low for a region of one second between
+        # pauses); power.draw.instant is a snapshot (no lag, several percent of noise)
+        watts, instant = under_load(2), under_load(7)
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx or None,
-                "reasons": sorted(reasons), "samples": len(sm), "watts": watts[len(watts) // 2] if watts else None}
+                "reasons": sorted(reasons), "samples": len(sm), "watts": watts, "watts_instant": instant}
 
 
 def workload_desc(name, groups=1, cap_b=0, cap_iters=100, fuse_gather=False):
@@ -428,11 +444,13 @@ def run_gpu(args):
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
             "saved_bytes": int(B.ec_saved_bytes(cfg)),
             "layer_tflops": (fl["fwd"] + fl["bwd"]) / (ms_step * 1e-3) / 1e12,
-            # under the board's power cap a step costs what it costs in energy: watts (median of the samples taken
-            # under load) x time per step; per flop of the layer it compares with the vendor's large square product
+            # under the board's power cap a step costs what it costs in energy: watts (mean of the samples taken
+            # under load; the unaveraged reading where nvidia-smi has one, a timed region being too short for the averaged one) x time per step; per flop of the layer it compares with the vendor's large square product
             # (`--gemms --loop-seconds`)
-            "energy": (lambda w: {"watts": w, "joules_per_step": round(w * ms_step * 1e-3, 3),
-                                  "pj_per_flop": round(w * ms_step * 1e-3 / (fl["fwd"] + fl["bwd"]) * 1e12, 4)} if w else None)(clocks.summary()["watts"]),
+            "energy": (lambda c: (lambda w: {"watts": w, "source": "power.draw.instant" if c["watts_instant"] else "power.draw",
+                                             "joules_per_step": round(w * ms_step * 1e-3, 3),
+                                             "pj_per_flop": round(w * ms_step * 1e-3 / (fl["fwd"] + fl["bwd"]) * 1e12, 4)} if w else None)
+                       (c["watts_instant"] or c["watts"]))(clocks.summary()),
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
@@ -641,7 +659,7 @@ def run_gemms(args):
 
     if args.loop_seconds > 0:
         # Energy view: every product loops for --loop-seconds, long enough for the power controller to settle and for
-        # nvidia-smi to sample power and clocks; energy per flop = median watts x time per call / flops.  A large square
+        # nvidia-smi to sample power and clocks; energy per flop = mean watts under load x time per call / flops.  A large square
         # product of the vendor library (nothing but tensor-core work, hardly any HBM traffic) calibrates the scale.
         side = 8192
         Sa, Sb, Sc = (torch.randn(side, side, device=dev, dtype=bf) for _ in range(3))
@@ -656,7 +674,7 @@ def run_gemms(args):
             with ClockSampler(torch.cuda.current_device()) as cs:
                 ms = timed(fn, count)
             c = cs.summary()
-            res.setdefault(name, {})[tag] = {"tflops": round(fl / ms / 1e9, 1), "ms": round(ms, 4), "sm_mhz": c["sm_mhz"], "watts": c["watts"],
+            res.setdefault(name, {})[tag] = {"tflops": round(fl / ms / 1e9, 1), "ms": round(ms, 4), "sm_mhz": c["sm_mhz"], "watts": c["watts"], "watts_instant": c["watts_instant"],
                                              "pj_per_flop": round(c["watts"] * ms * 1e-3 / fl * 1e12, 4) if c["watts"] else None,
                                              "reasons": c["reasons"]}
             time.sleep(0.5)
