@@ -412,6 +412,21 @@ def run_gpu(args):
     gemm_avg_ms = sum(gemm_ms) / max(1, len(gemm_ms))
     achieved = fl["gemm"] / (gemm_avg_ms * 1e-3) / 1e12 if gemm_ms else None
     peak = peaks["tflops_sustained"]
+    # This box's own sustained matmul rate, taken after all timed work with the vendor library (an 8192-cubed bf16 product in
+    # a loop of about a second and a half, the kind of loop the pool's peak figure comes from).  Context for the fraction
+    # above: the boxes of the pool differ by more than ten percent under the same power cap.  Calibration only.
+    box_peak = None
+    if world == 1 and args.workload == "cfg4" and not args.graph:
+        a8, b8, c8 = (torch.randn(8192, 8192, device=dev, dtype=bf) for _ in range(3))
+        for _ in range(20):
+            torch.mm(a8, b8, out=c8)
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(); q0.record()
+        for _ in range(1800):
+            torch.mm(a8, b8, out=c8)
+        q1.record(); torch.cuda.synchronize()
+        box_peak = 1800 * 2.0 * 8192 ** 3 / (q0.elapsed_time(q1) * 1e-3) / 1e12
+        del a8, b8, c8
 
     if rank == 0:
         cpu = None
@@ -439,6 +454,7 @@ def run_gpu(args):
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": (achieved / peak) if achieved else None,
                          "frac_of_nominal": (achieved / NOMINAL_BF16_TFLOPS) if achieved else None,
+                         "box_matmul_tflops": box_peak, "frac_of_box_matmul": (achieved / box_peak) if achieved and box_peak else None,
                          "peak_source": f"{peaks['source']} bf16 matmul, sustained", "traffic": gemm_traffic(args.workload, E),
                          "flops_per_launch": fl["gemm"], "avg_launch_ms": gemm_avg_ms},
             "stage_ms": {k_: round(v_, 4) for k_, v_ in stage_ms.items()},
