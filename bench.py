@@ -355,7 +355,7 @@ def run_gpu(args):
     # the stages are timed in the same sustained (power-capped) state as `value`.
     B.ec_profile_enable(True)
     stage_ms = {}
-    bursts, burst_steps = 3, max(2, min(args.steps, 10))
+    bursts, burst_steps = 6, max(2, min(args.steps, 10))
     plain_step = eager_step if args.graph else step         # the stage events are recorded at launch time
     for _ in range(bursts):
         for _ in range(burst_steps):
