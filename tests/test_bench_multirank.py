@@ -47,3 +47,23 @@ def test_reference_arm_prints_one_json_line_on_rank0_only():
     j = json.loads(out.stdout.strip().splitlines()[-1])
     assert j["impl"] == "reference" and j["cpu_baseline"]["kind"] == "oracle" and j["value"] > 0
     assert j["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_clock_sampler_summary_separates_load_from_idle_and_the_two_power_readings():
+    """The summary of the nvidia-smi samples: median clock, throttle reasons, power as the mean of the samples taken
+    under load, the averaged and the unaveraged reading kept apart, and nothing when there are no samples."""
+    sys.path.insert(0, ROOT) if ROOT not in sys.path else None
+    import bench
+    s = bench.ClockSampler.__new__(bench.ClockSampler)
+    idle = ["1965", "1965", "190.0", "Not Active", "Not Active", "Not Active", "Not Active"]
+    load = ["1260", "1965", "900.0", "Not Active", "Not Active", "Not Active", "Active"]
+    s.rows = [idle, load, load, load]
+    out = s.summary()
+    assert out["sm_mhz"] == 1260.0 and out["sm_max_mhz"] == 1965.0 and out["reasons"] == ["sw_power_cap"]
+    assert out["watts"] == 900.0 and out["watts_instant"] is None and out["samples"] == 4
+    s.rows = [idle + ["200.0"], load + ["1010.0"], load + ["990.0"]]
+    out = s.summary()
+    assert out["watts"] == 900.0 and out["watts_instant"] == 1000.0
+    s.rows = []
+    out = s.summary()
+    assert out["sm_mhz"] is None and out["watts"] is None and out["watts_instant"] is None and out["reasons"] == []
